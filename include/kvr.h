@@ -335,6 +335,14 @@ kvr_status_t kvr_reconstruct(const kvr_sketch_t* sk, int32_t layer, float* Kt, f
 /* N and R recorded by the last compress of a layer (host ints); STATE if never compressed. */
 kvr_status_t kvr_layer_shape(const kvr_sketch_t* sk, int32_t layer, int32_t* N, int32_t* R);
 
+/* Calibration, not part of the method: measures on the current device the two on-chip rates that
+ * bound Algorithm 2's reconstruction (the Vague Sketch section's element-wise median of r cells) --
+ * fp32 min/max operations per second (peaks[0], lane operations: one min or max of one element) with a
+ * register-only loop, and shared-memory bytes read per second (peaks[1]) with conflict-free 16-byte
+ * loads.  peaks: host [2], out.  Synchronous: launches two short kernels on `cuda_stream`, waits for
+ * them and returns; allocates and frees 512 bytes of device memory.  Errors: INVALID_ARG, ALLOC, CUDA. */
+kvr_status_t kvr_measure_pipe_peaks(double* peaks, void* cuda_stream);
+
 /* Number of kernels this library has launched on behalf of the handle since creation. */
 int64_t kvr_launch_count(const kvr_sketch_t* sk);
 

@@ -31,6 +31,7 @@ EXPORTS = (
     "kvr_sketch_set_decode_kernel", "kvr_last_decode_kernel", "kvr_sketch_device_status",
     "kvr_accumulate_scores", "kvr_demote", "kvr_sketch_set_score_kernel", "kvr_last_score_kernel",
     "kvr_accumulate_vague_scores", "kvr_swap", "kvr_sketch_set_obs_window_causal", "kvr_paper_storage_split", "kvr_layer_budgets", "kvr_sketch_set_combine",
+    "kvr_measure_pipe_peaks",
 )
 
 
@@ -93,6 +94,7 @@ def lib() -> ctypes.CDLL:
         L.kvr_last_score_kernel.restype = i32
         L.kvr_last_decode_kernel.argtypes = [vp]
         L.kvr_last_decode_kernel.restype = i32
+        L.kvr_measure_pipe_peaks.argtypes = [ctypes.POINTER(ctypes.c_double), vp]
         L.kvr_status_string.argtypes = [i32]
         L.kvr_status_string.restype = ctypes.c_char_p
         _lib = L
@@ -230,6 +232,13 @@ def kvr_sketch_set_obs_window_causal(sk: Sketch, on: bool):
 
 def kvr_last_score_kernel(sk: Sketch) -> int:
     return int(lib().kvr_last_score_kernel(sk.handle))
+
+
+def kvr_measure_pipe_peaks(stream=None):
+    """(fp32 min/max lane-ops per second, shared-memory bytes read per second) measured on the current device."""
+    out = (ctypes.c_double * 2)()
+    _check(lib().kvr_measure_pipe_peaks(out, _stream(stream)), "kvr_measure_pipe_peaks")
+    return float(out[0]), float(out[1])
 
 
 def kvr_launch_count(sk: Sketch) -> int:

@@ -4,9 +4,10 @@
 //
 // A compressed token J needs the element-wise median of three cells (Algorithm 2),
 //     K~_J[d] = med_i cellK[i][h_i(J)][d],     V~_J[d] = med_i g_i(J) cellV[i][h_i(J)][d],
-// i.e. 3 KB of fp32 cell data fetched from three random places.  On-chip traffic and the min/max
-// arithmetic of the medians, not HBM bytes, are what this costs, so the kernel is organised around
-// keeping cell reads on chip without any exchange between CTAs:
+// i.e. 3 KB of fp32 cell data fetched from three random places.  On-chip traffic, the min/max
+// arithmetic of the medians and the instruction issue slots around them, not HBM bytes, are what this
+// costs, so the kernel is organised around keeping cell reads on chip without any exchange between
+// CTAs, and around keeping little state per lane so that many warps are resident:
 //
 //   * The compressed tokens of a head-instance are grouped into C x C classes by
 //     (h_1(J) mod C, h_2(J) mod C).  All tokens of class (i, j) only touch the row-1 cells with
@@ -15,20 +16,24 @@
 //     the class's token entries once (bulk copies that report to an mbarrier; the wait on it is
 //     bounded) and serves the whole class, or a slice of it, from there.
 //   * Inside a class the tokens are ordered by their row-0 cell.  The row-0 cell of the current run
-//     of tokens stays in registers; the next run's cell is prefetched (cp.async) into a two-slot
-//     ring per group while the current run is processed.
+//     of tokens stays in registers; the next run's cell (named by the entry that starts the run) is
+//     fetched (cp.async) into the group's ring slot while the current run is processed.
 //   * A group of 16 lanes takes one token at a time: each lane owns 8 channels (4 + 4, so that the
-//     group reads 256 contiguous bytes of a cell per load, conflict-free), computes the medians with
-//     min/max, the G partial dot products with packed two-wide fp32 FMAs, and the 16 lanes add the
-//     partial logits with a transposing shuffle tree that leaves every lane with one head's logit.
-//   * While the cell slices are still in flight each group first streams its share of the retained
-//     rows (exact K/V, Algorithm 4's R.get / C.get) through the same accumulate routine, so one
-//     online-softmax state per group covers both kinds of token.  SMs that the class grid leaves idle
-//     run CTAs that only stream retained rows.
-//   * The running maximum of the online softmax is only raised when a logit exceeds it by 2^20
-//     (the weights stay far inside fp32 range), which keeps the rescale branch out of the loop.
+//     group reads 256 contiguous bytes of a cell per load, conflict-free).
+//   * The work is done in two passes over the CTA's tokens (retained rows and compressed tokens alike):
+//       key pass    a lane holds the scaled queries only; per token: medians of the key halves, the G
+//                   partial dot products with packed two-wide fp32 FMAs, a select-free transposing
+//                   shuffle tree (the lanes keep their queries in a head order permuted by lane, so
+//                   every level sends a fixed half), the logit goes to shared memory;
+//       weights     the CTA's maximum per head is known, so every logit becomes its softmax weight
+//                   (sign g_0 of a reconstructed token folded in) in place, and the sum is formed;
+//       value pass  a lane holds the output accumulators only; per token: medians of the value halves
+//                   and G packed multiply-adds with the weights read back from shared memory.
+//     Neither pass carries both the queries and the accumulators, there is no running maximum and no
+//     rescaling inside the loops, and the groups of a CTA are merged by plain sums in a fixed order.
 //   * Each CTA leaves one record (max, sum, o[G][128]); the last CTA of the head-instance to arrive
 //     merges the records.  Nothing in this kernel waits on another CTA.
+//   * SMs that the class grid leaves idle run CTAs that only stream retained rows.
 #include <type_traits>
 
 #include "kvr_decode_common.cuh"
@@ -37,16 +42,21 @@ namespace {
 using namespace kvr_dec;
 typedef unsigned long long u64;
 
-constexpr int NGRP = 32;            // token groups per CTA
-constexpr int KVR_LPT = 16;         // lanes per token group (16: 8 channels per lane, 512 threads)
+constexpr int LPT = 16;             // lanes per token group: 8 channels per lane
+constexpr int NT = 640;             // threads per CTA (at most 102 registers each)
+constexpr int NGRP = NT / LPT;      // token groups per CTA
+constexpr int NW = NT / 32;
+constexpr int NC = 32 / LPT;        // 16-byte chunks (4 channels) per lane and vector
+constexpr int NP = 2 * NC;          // packed pairs per lane and vector
+constexpr int DPL = 4 * NC;         // channels per lane
 constexpr int CELLF = 2 * KVR_D;    // floats of one staged cell: keys[128] | values[128]
 constexpr int CELLB = CELLF * 4;
+constexpr int HALFB = KVR_D * 4;    // bytes of the key half (or the value half) of a cell
 constexpr unsigned FULL = 0xFFFFFFFFu;
-constexpr float RESCALE_GAP = 20.f;
-constexpr size_t SMEM_LIMIT = 227 * 1024 - 512;   // dynamic part; the kernel also has a few hundred bytes of static shared memory
+constexpr size_t SMEM_LIMIT = 227 * 1024 - 1024;   // dynamic part; the kernel also has some static shared memory
 // time of one retained row relative to one reconstructed token (measured): in a CTA that also serves
-// a class (few rows, latency-bound) and in a CTA that only streams rows
-constexpr double COST_CLS = 1.0, COST_EXTRA = 0.63;
+// a class and in a CTA that only streams rows
+constexpr double COST_CLS = 0.45, COST_EXTRA = 0.45;
 
 struct StagedParams {
     const void* q;          // [n_inst][G][128]  16-bit
@@ -60,8 +70,11 @@ struct StagedParams {
     float* out;             // [n_inst][G][128]
     int* status;            // handle's device status word: bit 0 set when a bounded wait gave up
     float* ml;              // handle base: [inst][G][2] reference maximum and sum of the softmax
-    int inst0, R, b, C, logC, n1, max_ctx, S, lcap;
+    int inst0, R, b, C, logC, n1, max_ctx, S;
+    int lcap;               // token entries staged at a time
+    int rcap, rcap_extra;   // retained rows whose logits fit beside them (class CTAs / row-only CTAs)
     int n_ccta, r_cls;      // class CTAs per head-instance; retained rows they share (extra CTAs take the rest)
+    uint32_t zero;          // 0, unknown to the compiler (orders a shared-memory read before a copy into the same bytes)
     float scale_log2e;
 };
 
@@ -84,13 +97,20 @@ __device__ __forceinline__ void static_for(F&& f) {
         static_for<I + 1, N>(f);
     }
 }
-// the same for memory that does change (ring slots, token entries)
-template <int OFF>
+// the same for memory that does change (ring slots, token entries, weights)
 __device__ __forceinline__ float4 lds_vol(uint32_t addr) {
     float4 v;
-    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4+%5];\n"
-                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr), "n"(OFF) : "memory");
+    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];\n"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
     return v;
+}
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];\n" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts_f32(uint32_t addr, float v) {
+    asm volatile("st.shared.f32 [%0], %1;\n" ::"r"(addr), "f"(v) : "memory");
 }
 // ---- bulk copies global -> shared that report to an mbarrier ---------------------------------------
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -126,14 +146,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     }
     return true;
 }
-__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
-    uint32_t v;
-    asm volatile("ld.shared.u32 %0, [%1];\n" : "=r"(v) : "r"(addr) : "memory");
-    return v;
-}
 __device__ __forceinline__ uint2 ld_stream8(const uint2* p) {
     uint2 r;
     asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(p));
+    return r;
+}
+// a load the compiler must leave where it stands (the queries are read again for every stretch of
+// tokens instead of being kept in registers through the value pass)
+__device__ __forceinline__ uint2 ld_here8(const uint2* p) {
+    uint2 r;
+    asm volatile("ld.global.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(p) : "memory");
     return r;
 }
 // packed pairs of fp32 (sm_100 has two-wide fp32 multiply-add: half the issue slots)
@@ -169,453 +191,564 @@ __device__ __forceinline__ void unpack4(const uint2& x, u64 (&pr)[2]) {
 
 // Shared-memory carve-up, in bytes from the start of the dynamic segment (all multiples of 16).
 struct Layout {
-    int flag, ring, list, cells, total;
+    int ctrl, acc, ring, desc, stage, wbuf, cells, total;
 };
-__host__ __device__ inline Layout make_layout(int n1, int lcap) {
+// n1: cells per staged slice; lcap: token entries held at a time (even); rcap: retained rows whose
+// logits are kept beside them; G: query heads per kv head
+__host__ __device__ inline Layout make_layout(int n1, int lcap, int rcap, int G) {
     Layout L;
     int o = 0;
-    L.flag = o;  o += 16;                       // last-arriver flag (int) and, at +8, the staging mbarrier
-    L.ring = o;  o += NGRP * 2 * CELLB;         // per token group: two row-0 cells (also the merge scratch)
-    L.list = o;  o += ((lcap + 2) * 8 + 15) & ~15;   // staged token entries (+2: bulk copies move whole 16 bytes)
-    L.cells = o; o += 2 * n1 * CELLB;           // row-1 slice, then row-2 slice
+    L.ctrl = o;  o += 32;                            // last-arriver flag (int); at +16 and +24 the two staging mbarriers
+    L.acc = o;   o += (G * PART * 4 + 15) & ~15;     // the CTA's record while stretches of tokens are folded into it
+    L.ring = o;  o += NGRP * HALFB;                  // per token group: half of a row-0 cell in flight (also the merge scratch)
+    L.desc = o;                                      // one 16-byte descriptor per token entry; the 8-byte entries
+    L.stage = o + (lcap + 2) * 8;                    //   land in the upper half (+2: bulk copies move whole 16 bytes)
+    o += (lcap + 2) * 16;
+    L.wbuf = o;  o += ((rcap + lcap + 1) * G * 4 + 15) & ~15;   // one logit, later weight, per (token, head); + a zero slot
+    L.cells = o; o += 2 * n1 * CELLB;                // row-1 slice, then row-2 slice
     L.total = o;
     return L;
 }
 
-// LPT = lanes per token (a "group"); every CTA has NGRP groups, so NT = NGRP * LPT threads.
-// Lane l of a group owns the 16-byte channel chunks l, LPT + l, 2 LPT + l, ... of each 512-byte
-// vector, so that the LPT lanes of a group read LPT * 16 contiguous bytes with every load.
-// MEAN: the three cells of a token are averaged instead of the paper's element-wise median (an option
-// of the handle; the averages run on the two-wide fp32 multiply-add pipe).
-template <typename T, int G, int LPT, bool MEAN>
-__global__ void __launch_bounds__(NGRP * LPT, 1)
+// G: query heads per kv head.  MEAN: the three cells of a token are averaged instead of the paper's
+// element-wise median (an option of the handle; the averages run on the two-wide fp32 multiply-add pipe).
+template <typename T, int G, bool MEAN>
+__global__ void __launch_bounds__(NT, 1)
 decode_staged_kernel(const StagedParams p) {
-    constexpr int NT = NGRP * LPT, NW = NT / 32;
-    constexpr int NC = 32 / LPT;           // 16-byte chunks (4 channels) per lane and vector
-    constexpr int NP = 2 * NC;             // packed pairs per lane and vector
-    constexpr int DPL = 4 * NC;            // channels per lane
-    constexpr int LG = (LPT == 16) ? 4 : 3;
     constexpr int LOGG = (G == 4) ? 2 : (G == 2) ? 1 : 0;
-    constexpr int SH = LG - LOGG;          // lane (g << SH) of a group speaks for head g
+    constexpr int LGL = (LPT == 16) ? 4 : 3;
+    constexpr int SH = LGL - LOGG;         // lanes (g << SH) .. of a group end up with head g's logit
     static_assert(LPT == 16 || LPT == 8, "lanes per token");
+    static_assert(NT >= G * KVR_D && NT % 32 == 0 && NW <= 32, "one thread per (head, channel) folds the groups");
     extern __shared__ __align__(16) unsigned char smem[];
-    const Layout L = make_layout(p.n1, p.lcap);
-    int* s_flag = reinterpret_cast<int*>(smem + L.flag);
-    float* s_ring = reinterpret_cast<float*>(smem + L.ring);
-    uint2* s_list = reinterpret_cast<uint2*>(smem + L.list);
-    float* s_cells = reinterpret_cast<float*>(smem + L.cells);
+    // (g0 g1, g0 g1, g0 g2, g0 g2) for the 8 sign patterns of an entry; static shared memory sits at
+    // the bottom of the window, so the table's address fits the 16 bits a descriptor has for it
+    __shared__ __align__(128) float4 s_sign[8];
+    __shared__ float s_red[NW][4];
+    __shared__ float s_M[4], s_L[4];
 
+    const Layout L = make_layout(p.n1, p.lcap, p.rcap, G);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, grp = tid / LPT, lg = tid & (LPT - 1);
     const int u = blockIdx.y, inst = p.inst0 + u, b = p.b, C = p.C, n1 = p.n1;
     const int rec = blockIdx.x, n_rec = gridDim.x;
     const bool extra = rec >= p.n_ccta;            // a CTA that only streams retained rows
     const int cls = extra ? 0 : rec / p.S, sp = rec - cls * p.S;
     const int ci = cls >> p.logC, cj = cls & (C - 1);
-    __shared__ float4 s_sign[8];                   // (g0, g0 g1, g0 g2, -) for the 8 sign patterns of an entry
-    if (tid < 8) s_sign[tid] = make_float4((tid & 1) ? -1.f : 1.f, (tid & 2) ? -1.f : 1.f, (tid & 4) ? -1.f : 1.f, 0.f);
+    if (tid < 8) s_sign[tid] = make_float4((tid & 2) ? -1.f : 1.f, (tid & 2) ? -1.f : 1.f, (tid & 4) ? -1.f : 1.f, (tid & 4) ? -1.f : 1.f);
     // A following decode launch may be scheduled as soon as every CTA of this one is running: its
     // CTAs take the SMs this launch frees one by one and stage their cells while this launch drains.
     asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
 
-    // this CTA's slice of its class
-    const int32_t* coff = p.coff + (size_t)inst * (C * C + 1);
-    int s_begin = 0, s_end = 0;
+    const uint32_t smem_s = (uint32_t)__cvta_generic_to_shared(smem);
+    const uint32_t cells_s = smem_s + L.cells, desc_s = smem_s + L.desc, wbuf_s = smem_s + L.wbuf;
+    // ---------------------------------------------------------------- start staging.  The class's cells
+    // travel as bulk copies that report to one mbarrier, the first stretch of its token entries to a
+    // second one.  The cell copies need nothing but the class number, so they go first; a warp issues
+    // its copies one lane after the other, so they are dealt to the warps round-robin.
+    const uint32_t bar_cells = smem_s + L.ctrl + 16u, bar_list = smem_s + L.ctrl + 24u;
     if (!extra) {
-        const int k_lo = coff[cls], k_len = coff[cls + 1] - k_lo;
-        s_begin = k_lo + (int)((long long)k_len * sp / p.S);
-        s_end = k_lo + (int)((long long)k_len * (sp + 1) / p.S);
-    }
-    const uint2* clist = p.clist + (size_t)inst * p.max_ctx;
-    const float* cellsK = p.cells + (size_t)inst * 2 * KVR_R * b * KVR_D;
-    const float* cellsV = cellsK + (size_t)KVR_R * b * KVR_D;
-    const uint32_t cells_s = (uint32_t)__cvta_generic_to_shared(s_cells);
-
-    // ---------------------------------------------------------------- start staging: the class's cells and
-    // the first chunk of its token entries travel as bulk copies that report to one mbarrier
-    const uint32_t bar = (uint32_t)__cvta_generic_to_shared(smem + L.flag) + 8u;
-    const uint32_t list_base = (uint32_t)__cvta_generic_to_shared(s_list);
-    const int len0 = min(p.lcap, s_end - s_begin);
-    // a bulk copy starts on 16 bytes: take the entry before, if need be (entries are 8 bytes)
-    const int lshift = (int)(((size_t)inst * p.max_ctx + s_begin) & 1);
-    if (len0 > 0) {
+        const float* cellsK = p.cells + (size_t)inst * 2 * KVR_R * b * KVR_D;
+        const float* cellsV = cellsK + (size_t)KVR_R * b * KVR_D;
         if (tid == 0) {
-            mbar_init(bar, 1);
+            mbar_init(bar_cells, 1);
+            mbar_init(bar_list, 1);
             const int cnt1 = (b - ci + C - 1) >> p.logC, cnt2 = (b - cj + C - 1) >> p.logC;   // cells of the two slices
-            mbar_expect_tx(bar, (uint32_t)((cnt1 + cnt2) * CELLB + ((len0 + lshift + 1) & ~1) * 8));
+            mbar_expect_tx(bar_cells, (uint32_t)((cnt1 + cnt2) * CELLB));
         }
         __syncthreads();
-        for (int i = tid; i < 4 * n1; i += NT) {       // one 512-byte piece per (cell, keys | values)
+        for (int i = warp + lane * NW; i < 4 * n1; i += NT) {       // one 512-byte piece per (cell, keys | values)
             const int idx = i >> 1, kv = i & 1;
             const int h = (idx < n1) ? idx * C + ci : (idx - n1) * C + cj;
             const int row = (idx < n1) ? 1 : 2;
             if (h < b)
-                bulk_g2s(cells_s + (uint32_t)(idx * CELLB + kv * (KVR_D * 4)),
-                         (kv ? cellsV : cellsK) + ((size_t)row * b + h) * KVR_D, KVR_D * 4, bar);
+                bulk_g2s(cells_s + (uint32_t)(idx * CELLB + kv * HALFB),
+                         (kv ? cellsV : cellsK) + ((size_t)row * b + h) * KVR_D, HALFB, bar_cells);
         }
-        if (tid == NT - 1)
-            bulk_g2s(list_base, clist + (s_begin - lshift), (uint32_t)(((len0 + lshift + 1) & ~1) * 8), bar);
     }
-    // Each group asks for the row-0 cell of its first token right away (entry read from global memory).
-    const uint32_t ring_s = (uint32_t)__cvta_generic_to_shared(s_ring) + (uint32_t)(grp * 2 * CELLB + lg * 16);
-    auto fetch_row0 = [&](uint32_t c0, uint32_t slot) {      // row-0 cell c0 -> ring slot (this lane's pieces)
-        // (addresses rebuilt from the kernel arguments: this runs once per run of tokens, and keeping
-        // two 64-bit pointers alive through the token loop costs registers the loop needs)
-        const float* gk = p.cells + ((size_t)(p.inst0 + blockIdx.y) * 2 * KVR_R * p.b + c0) * KVR_D + 4 * lg;
-        const float* gv = gk + (size_t)KVR_R * p.b * KVR_D;
-        const uint32_t dst = ring_s + slot * CELLB;
-#pragma unroll
-        for (int c = 0; c < NC; ++c) {
-            cp_async16(dst + c * LPT * 16, gk + c * LPT * 4);
-            cp_async16(dst + 512 + c * LPT * 16, gv + c * LPT * 4);
+    // this CTA's slice of its class, and its retained rows
+    int s_begin = 0, s_end = 0, r_begin, r_end;
+    if (!extra) {
+        const int32_t* coff = p.coff + (size_t)inst * (C * C + 1);
+        const int k_lo = coff[cls], k_len = coff[cls + 1] - k_lo;
+        s_begin = k_lo + (int)((long long)k_len * sp / p.S);
+        s_end = k_lo + (int)((long long)k_len * (sp + 1) / p.S);
+        r_begin = (int)((long long)p.r_cls * rec / p.n_ccta);
+        r_end = (int)((long long)p.r_cls * (rec + 1) / p.n_ccta);
+    } else {
+        const int e = rec - p.n_ccta, n_e = n_rec - p.n_ccta, rest = p.R - p.r_cls;
+        r_begin = p.r_cls + (int)((long long)rest * e / n_e);
+        r_end = p.r_cls + (int)((long long)rest * (e + 1) / n_e);
+    }
+    const int lcap = p.lcap, rcap = extra ? p.rcap_extra : p.rcap;
+    const uint2* clist = p.clist + (size_t)inst * p.max_ctx;
+    const int len0 = min(lcap, s_end - s_begin);
+    // a bulk copy starts on 16 bytes: take the entry before, if need be (entries are 8 bytes)
+    const int lshift = (int)(((size_t)inst * p.max_ctx + s_begin) & 1);
+    if (len0 > 0 && tid == 0) {
+        const uint32_t bytes = (uint32_t)(((len0 + lshift + 1) & ~1) * 8);
+        mbar_expect_tx(bar_list, bytes);
+        bulk_g2s(smem_s + L.stage, clist + (s_begin - lshift), bytes, bar_list);
+    }
+    // The rows are read twice (keys, later values), microseconds apart: ask for all of them now, so
+    // that both reads find them in the L2 cache instead of waiting for HBM one batch at a time.
+    {
+        constexpr int PF = 8192;                            // bytes per prefetch request (32 rows)
+        const char* k8 = reinterpret_cast<const char*>(p.Kr + ((size_t)u * p.R + r_begin) * 32);
+        const char* v8 = reinterpret_cast<const char*>(p.Vr + ((size_t)u * p.R + r_begin) * 32);
+        const int bytes = (r_end - r_begin) * 256;
+        for (int o = (warp + lane * NW) * PF; o < bytes; o += NT * PF) {     // (dealt to the warps like the cell copies)
+            const uint32_t n = (uint32_t)min(PF, bytes - o);
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(k8 + o), "r"(n) : "memory");
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(v8 + o), "r"(n) : "memory");
         }
+    }
+    // stretches: the tokens are taken lcap entries and rcap rows at a time (normally all at once)
+    int n_str = 1;
+    {
+        const int a_ = (s_end - s_begin + lcap - 1) / lcap, b_ = (r_end - r_begin + rcap - 1) / rcap;
+        n_str = max(1, max(a_, b_));
+    }
+    const uint32_t wzero_s = wbuf_s + (uint32_t)(extra ? p.rcap_extra : p.rcap + lcap) * (G * 4);
+    const uint32_t sign_s = (uint32_t)__cvta_generic_to_shared(s_sign);
+    float* s_acc = reinterpret_cast<float*>(smem + L.acc);
+    // Row-0 cells: each lane moves its own 16-byte pieces of the key half or the value half of a cell
+    // into its group's ring slot, and later reads exactly those bytes back.  g0 = this lane's piece of
+    // that half of row-0 cell 0.
+    const uint32_t ring_s = smem_s + L.ring + (uint32_t)(grp * HALFB + lg * 16);
+    auto fetch_row0 = [&](const float* g0, uint32_t c0, uint32_t z) {
+        const float* g = g0 + (size_t)c0 * KVR_D;
+#pragma unroll
+        for (int c = 0; c < NC; ++c) cp_async16(ring_s + z + c * LPT * 16, g + c * LPT * 4);
         asm volatile("cp.async.commit_group;\n" ::);
     };
+    // Take the fetched half cell into registers and ask for the next run's.  The copy must not start
+    // before the bytes are read: its address is made to depend on the loaded values (z is always 0).
+    auto switch_run = [&](float (&r0v)[DPL], const float* g0, uint32_t c0_next) {
+        asm volatile("cp.async.wait_all;\n" ::: "memory");
+        uint32_t z = 0;
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+            const float4 a = lds_vol(ring_s + c * LPT * 16);
+            r0v[4 * c] = a.x; r0v[4 * c + 1] = a.y; r0v[4 * c + 2] = a.z; r0v[4 * c + 3] = a.w;
+            z |= __float_as_uint(a.w);
+        }
+        fetch_row0(g0, c0_next, z & p.zero);
+    };
+    // the group's share of a stretch of `len` entries: the first rn groups take qn + 1 tokens, the others qn
+    auto share = [&](int len, int& qn, int& rn, int& r0) {
+        qn = len / NGRP;
+        rn = len - qn * NGRP;
+        r0 = grp * qn + min(grp, rn);
+    };
+    // Each group asks for the row-0 key half of its first token right away (entry read from global memory).
+    uint32_t c0_first = 0;
     if (len0 > 0) {
-        const int qn = len0 / NGRP, rn = len0 - qn * NGRP;
-        if (qn + (grp < rn ? 1 : 0) > 0)
-            fetch_row0(clist[s_begin + grp * qn + min(grp, rn)].y >> KVR_CL_C0_SHIFT, 0);
+        int qn, rn, r0;
+        share(len0, qn, rn, r0);
+        if (qn + (grp < rn ? 1 : 0) > 0) {
+            c0_first = clist[s_begin + r0].y >> KVR_CL_C0_SHIFT;
+            fetch_row0(p.cells + (size_t)inst * 2 * KVR_R * b * KVR_D + 4 * lg, c0_first, 0u);
+        }
     }
 
-    // ---------------------------------------------------------------- everything above reads only what no
-    // decode launch writes (cells, token lists).  When this launch was made a programmatic dependent
-    // of the previous decode launch, it may have started while that one was still running: wait for
-    // it here, before the queries are read and before anything is written to global memory.
-    asm volatile("griddepcontrol.wait;\n" ::: "memory");
-    // ---------------------------------------------------------------- the queries: the retained rows need them
-    // while the cell slices are still on their way.  After the shuffle tree lane lg holds the logit
-    // of head lg >> SH.
-    const int own = lg >> SH;
-    u64 q2[G][NP];
-    {
-        const uint2* qg = reinterpret_cast<const uint2*>(p.q) + (size_t)u * G * 32;     // 32 8-byte pieces per head
-        const u64 sc2 = pack2(p.scale_log2e, p.scale_log2e);
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-#pragma unroll
-            for (int c = 0; c < NC; ++c) {
-                u64 t2[2];
-                unpack4<T>(qg[g * 32 + c * LPT + lg], t2);
-                q2[g][2 * c] = mul2(t2[0], sc2);
-                q2[g][2 * c + 1] = mul2(t2[1], sc2);
+    const int own = lg >> SH;                                  // the head whose logit this lane ends up with
+    const uint32_t lane16 = (uint32_t)(lg * 16);
+
+    for (int st = 0; st < n_str; ++st) {
+        const int rb = min(r_begin + st * rcap, r_end), re = min(rb + rcap, r_end), nrows = re - rb;
+        const int cb = min(s_begin + st * lcap, s_end), len = min(lcap, s_end - cb);
+        int qn, rn, r0;
+        share(len, qn, rn, r0);
+        const bool ragged_live = grp < rn;                     // this group has a token in the ragged last round
+        if (st > 0) {
+            __syncthreads();                                   // previous stretch consumed
+            asm volatile("cp.async.wait_all;\n" ::: "memory");
+            if (qn + (ragged_live ? 1 : 0) > 0) {
+                c0_first = clist[cb + r0].y >> KVR_CL_C0_SHIFT;
+                fetch_row0(p.cells + (size_t)inst * 2 * KVR_R * b * KVR_D + 4 * lg, c0_first, 0u);
             }
         }
-    }
-    float m_own = M_EMPTY, l_own = 0.f;
-    u64 o2[G][NP];
-#pragma unroll
-    for (int g = 0; g < G; ++g)
-#pragma unroll
-        for (int k = 0; k < NP; ++k) o2[g][k] = 0ull;
-
-    // one token: kp / vp = its key / value on this lane's channels, wsign = +1 or -1 (g_0 of a
-    // reconstructed token), valid = false for the filler token of a ragged last round
-    auto accumulate = [&](const u64 (&kp)[NP], const u64 (&vp)[NP], float wsign, bool valid) {
-        float s[G];
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-            u64 acc = mul2(q2[g][0], kp[0]);
-#pragma unroll
-            for (int k = 1; k < NP; ++k) acc = fma2(q2[g][k], kp[k], acc);
-            float lo, hi;
-            unpack2(acc, lo, hi);
-            s[g] = lo + hi;
-        }
-        // add over the lanes of the group; the first log2(G) levels hand half of the heads to the
-        // partner, so that lane lg ends with the complete logit of head lg >> SH
-        constexpr int X1 = LPT / 2, X2 = LPT / 4;
-        float mine;
-        if constexpr (G == 4) {
-            const bool hi1 = (lg & X1) != 0, hi2 = (lg & X2) != 0;
-            float k0_ = hi1 ? s[2] : s[0], k1_ = hi1 ? s[3] : s[1];
-            k0_ += __shfl_xor_sync(FULL, hi1 ? s[0] : s[2], X1);
-            k1_ += __shfl_xor_sync(FULL, hi1 ? s[1] : s[3], X1);
-            mine = hi2 ? k1_ : k0_;
-            mine += __shfl_xor_sync(FULL, hi2 ? k0_ : k1_, X2);
-        } else if constexpr (G == 2) {
-            const bool hi1 = (lg & X1) != 0;
-            mine = hi1 ? s[1] : s[0];
-            mine += __shfl_xor_sync(FULL, hi1 ? s[0] : s[1], X1);
-            mine += __shfl_xor_sync(FULL, mine, X2);
-        } else {
-            mine = s[0];
-            mine += __shfl_xor_sync(FULL, mine, X1);
-            mine += __shfl_xor_sync(FULL, mine, X2);
-        }
-#pragma unroll
-        for (int x = LPT / 8; x >= 1; x >>= 1) mine += __shfl_xor_sync(FULL, mine, x);
-        const bool grow = valid && (mine > m_own + RESCALE_GAP);
-        if (__any_sync(FULL, grow)) {
-            const float m_new = grow ? mine : m_own;
-            const float c = ex2(m_own - m_new);
-            l_own *= c;
-            m_own = m_new;
+        // ------------------------------------------------------------ key pass
+        // The scaled queries, head order permuted by lane: slot i holds head i ^ own, so that every
+        // level of the shuffle tree below keeps its low slots and sends its high slots.
+        u64 q2[G][NP];
+        {
+            const uint2* qg = reinterpret_cast<const uint2*>(p.q) + (size_t)u * G * 32;     // 32 8-byte pieces per head
+            const u64 sc2 = pack2(p.scale_log2e, p.scale_log2e);
 #pragma unroll
             for (int g = 0; g < G; ++g) {
-                const float cg = __shfl_sync(FULL, c, g << SH, LPT);
-                const u64 c2 = pack2(cg, cg);
-#pragma unroll
-                for (int k = 0; k < NP; ++k) o2[g][k] = mul2(o2[g][k], c2);
-            }
-        }
-        const float pr = valid ? ex2(mine - m_own) : 0.f;
-        l_own += pr;
-        const float pv_own = pr * wsign;
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-            const float pv = __shfl_sync(FULL, pv_own, g << SH, LPT);
-            const u64 pv2 = pack2(pv, pv);
-#pragma unroll
-            for (int k = 0; k < NP; ++k) o2[g][k] = fma2(pv2, vp[k], o2[g][k]);
-        }
-    };
-
-    // ---------------------------------------------------------------- retained tokens (exact rows)
-    {
-        int r_begin, r_end;
-        if (!extra) {
-            r_begin = (int)((long long)p.r_cls * rec / p.n_ccta);
-            r_end = (int)((long long)p.r_cls * (rec + 1) / p.n_ccta);
-        } else {
-            const int e = rec - p.n_ccta, n_e = n_rec - p.n_ccta, rest = p.R - p.r_cls;
-            r_begin = p.r_cls + (int)((long long)rest * e / n_e);
-            r_end = p.r_cls + (int)((long long)rest * (e + 1) / n_e);
-        }
-        const uint2* Kr = p.Kr + (size_t)u * p.R * 32 + lg;
-        const uint2* Vr = p.Vr + (size_t)u * p.R * 32 + lg;
-        constexpr int FL = (LPT == 16) ? 4 : 2;                    // tokens per group in flight
-        for (int base = r_begin; base < r_end; base += FL * NGRP) {
-            uint2 kx[FL][NC], vx[FL][NC];
-            bool ok[FL];
-#pragma unroll
-            for (int i = 0; i < FL; ++i) {
-                const int t = base + i * NGRP + grp;
-                ok[i] = t < r_end;
-                const size_t tt = (size_t)(ok[i] ? t : r_begin) * 32;
 #pragma unroll
                 for (int c = 0; c < NC; ++c) {
-                    kx[i][c] = ld_stream8(Kr + tt + c * LPT);
-                    vx[i][c] = ld_stream8(Vr + tt + c * LPT);
+                    u64 t2[2];
+                    unpack4<T>(ld_here8(qg + (g ^ own) * 32 + c * LPT + lg), t2);
+                    q2[g][2 * c] = mul2(t2[0], sc2);
+                    q2[g][2 * c + 1] = mul2(t2[1], sc2);
                 }
-            }
-#pragma unroll
-            for (int i = 0; i < FL; ++i) {
-                u64 kp[NP], vp[NP], t2[2];
-#pragma unroll
-                for (int c = 0; c < NC; ++c) {
-                    unpack4<T>(kx[i][c], t2); kp[2 * c] = t2[0]; kp[2 * c + 1] = t2[1];
-                    unpack4<T>(vx[i][c], t2); vp[2 * c] = t2[0]; vp[2 * c + 1] = t2[1];
-                }
-                accumulate(kp, vp, 1.f, ok[i]);
             }
         }
-    }
-
-    // ---------------------------------------------------------------- compressed tokens of the class slice
-    const uint32_t lane_cells = cells_s + (uint32_t)(lg * 16);
-    if (len0 > 0 && !mbar_wait(bar, 0)) atomicOr(p.status, 1);       // cells and first entries have landed
-    for (int c_begin = s_begin; c_begin < s_end; c_begin += p.lcap) {     // normally a single chunk
-        const int len = min(p.lcap, s_end - c_begin);
-        const bool first_chunk = c_begin == s_begin;
-        const int loff = first_chunk ? lshift : 0;
-        const uint32_t list_s = list_base + (uint32_t)loff * 8u;           // shared address of entry 0 of the chunk
-        if (!first_chunk) {
-            __syncthreads();                      // previous chunk consumed
-            for (int i = tid; i < len; i += NT) s_list[i] = clist[c_begin + i];
+        // logit (log2 units) of head `own` for the token whose key channels are kp
+        auto logit = [&](const u64 (&kp)[NP]) -> float {
+            float s[G];
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                u64 acc = mul2(q2[g][0], kp[0]);
+#pragma unroll
+                for (int k = 1; k < NP; ++k) acc = fma2(q2[g][k], kp[k], acc);
+                float lo, hi;
+                unpack2(acc, lo, hi);
+                s[g] = lo + hi;
+            }
+            float mine;
+            if constexpr (G == 4) {
+                const float t0 = s[0] + __shfl_xor_sync(FULL, s[2], LPT / 2);
+                const float t1 = s[1] + __shfl_xor_sync(FULL, s[3], LPT / 2);
+                mine = t0 + __shfl_xor_sync(FULL, t1, LPT / 4);
+#pragma unroll
+                for (int x = LPT / 8; x >= 1; x >>= 1) mine += __shfl_xor_sync(FULL, mine, x);
+            } else if constexpr (G == 2) {
+                mine = s[0] + __shfl_xor_sync(FULL, s[1], LPT / 2);
+#pragma unroll
+                for (int x = LPT / 4; x >= 1; x >>= 1) mine += __shfl_xor_sync(FULL, mine, x);
+            } else {
+                mine = s[0];
+#pragma unroll
+                for (int x = LPT / 2; x >= 1; x >>= 1) mine += __shfl_xor_sync(FULL, mine, x);
+            }
+            return mine;
+        };
+        constexpr int FLB = (LPT == 16) ? 8 : 4, FLT = (LPT == 16) ? 2 : 1;                            // rows per group in flight: full blocks, tail
+        // retained rows (exact keys): row t of the stretch goes to group t mod NGRP.  All lanes of a
+        // (token, head) quad hold the same logit and store it to the same word.
+        if (nrows > 0) {
+            const uint2* Kr = p.Kr + ((size_t)u * p.R + rb) * 32 + lg;
+            const uint32_t wb0 = wbuf_s + (uint32_t)(own * 4);
+            auto rows_key = [&](auto FLc, auto CHK, int base) {
+                constexpr int FLn = decltype(FLc)::value;
+                constexpr bool CHECK = decltype(CHK)::value;
+                const uint2* kb = Kr + (size_t)(base + grp) * 32;
+                uint2 kx[FLn][NC];
+#pragma unroll
+                for (int i = 0; i < FLn; ++i) {
+                    const bool ok = !CHECK || base + i * NGRP + grp < nrows;
+#pragma unroll
+                    for (int c = 0; c < NC; ++c) kx[i][c] = ld_stream8((ok ? kb + i * NGRP * 32 : Kr) + c * LPT);
+                }
+                const uint32_t wb = wb0 + (uint32_t)(base + grp) * (G * 4);
+#pragma unroll
+                for (int i = 0; i < FLn; ++i) {
+                    u64 kp[NP], t2[2];
+#pragma unroll
+                    for (int c = 0; c < NC; ++c) { unpack4<T>(kx[i][c], t2); kp[2 * c] = t2[0]; kp[2 * c + 1] = t2[1]; }
+                    const float mine = logit(kp);
+                    if (!CHECK || base + i * NGRP + grp < nrows) sts_f32(wb + i * NGRP * G * 4, mine);
+                }
+            };
+            int base = 0;
+            for (; base + FLB * NGRP <= nrows; base += FLB * NGRP) rows_key(std::integral_constant<int, FLB>{}, std::false_type{}, base);
+            for (; base < nrows; base += FLT * NGRP) rows_key(std::integral_constant<int, FLT>{}, std::true_type{}, base);
+        }
+        // ------------------------------------------------------------ token entries -> descriptors
+        // One thread per entry turns the 8-byte entry into what the two token loops need without further
+        // arithmetic: x, y = shared addresses of its row-1 and row-2 cells, z = address of its logit /
+        // weight slot, w = row-0 cell of the next run << 16 | address of its sign pairs | run flag
+        // (also set for the first token of every group).  The entries lie in the upper half of the
+        // descriptor array; a batch of descriptors only overwrites entries that were read before.
+        if (st == 0 && len0 > 0 && !mbar_wait(bar_list, 0)) atomicOr(p.status, 1);       // the first entries have landed
+        {
+            const uint2* staged = reinterpret_cast<const uint2*>(smem + L.stage) + lshift;
+            uint4* desc = reinterpret_cast<uint4*>(smem + L.desc);
+            const int split = rn * (qn + 1);
+            for (int base = 0; base < len; base += NT) {
+                const int i = base + tid;
+                uint2 e = make_uint2(0u, 0u);
+                if (i < len) e = (st == 0) ? staged[i] : clist[cb + i];
+                __syncthreads();
+                if (i < len) {
+                    bool start = true;                         // first token of its group?
+                    if (qn > 0) start = (i < split) ? (i % (qn + 1) == 0) : ((i - split) % qn == 0);
+                    uint4 d;
+                    d.x = cells_s + (e.x & 0xFFu) * CELLB;
+                    d.y = cells_s + ((e.x >> 8) & 0xFFu) * CELLB;
+                    d.z = wbuf_s + (uint32_t)(nrows + i) * (G * 4);
+                    d.w = (e.x & 0xFFFF0000u) | (sign_s + (e.y & 0x70u)) | (e.y & KVR_CL_FLAG) | (start ? KVR_CL_FLAG : 0u);
+                    desc[i] = d;
+                }
+            }
             __syncthreads();
         }
-        // the groups take contiguous runs: the first rn of them qn + 1 tokens, the others qn
-        const int qn = len / NGRP, rn = len - qn * NGRP;
-        const int r0 = grp * qn + min(grp, rn);
-        const int cnt = qn + (grp < rn ? 1 : 0);
-        const int r1 = r0 + cnt;
-
-        float k0[DPL], v0[DPL];                   // row-0 cell of the current run (this lane's channels)
+        const float* g0K = p.cells + (size_t)inst * 2 * KVR_R * b * KVR_D + 4 * lg;
+        if (st == 0 && !extra && !mbar_wait(bar_cells, 0)) atomicOr(p.status, 1);       // the cells have landed
+        // compressed tokens (Algorithm 2 on the key halves)
+        if (len > 0) {
+            float k0[DPL];                                // key half of the run's row-0 cell (this lane's channels)
 #pragma unroll
-        for (int x = 0; x < DPL; ++x) { k0[x] = 0.f; v0[x] = 0.f; }
-        uint32_t cur = 0;
-        if (!first_chunk && cnt > 0) fetch_row0(lds_u32(list_s + (uint32_t)r0 * 8u + 4u) >> KVR_CL_C0_SHIFT, 0);
-
-        // Reconstruction of one token (Algorithm 2 on this lane's channels): lp = shared address of
-        // its entry; force = the group's first token (its row-0 cell is needed whether or not the entry
-        // starts a run); live = false for the filler token of a ragged last round.
-        auto reconstruct = [&](uint32_t lp, bool live, bool force, u64 (&kp)[NP], u64 (&vp)[NP], float& wsign) {
-            uint2 e;
-            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];\n" : "=r"(e.x), "=r"(e.y) : "r"(lp) : "memory");
-            if (live && ((e.y & KVR_CL_FLAG) || force)) {
-                // a new run of tokens sharing one row-0 cell: take the prefetched cell into registers
-                // (the group's lane mask is rebuilt here: this branch is rare and the loop is short of registers)
-                const unsigned gmask = ((LPT == 16) ? 0xFFFFu : 0xFFu) << ((threadIdx.x & 31) & (32 - LPT));
-                asm volatile("cp.async.wait_all;\n" ::: "memory");
-                __syncwarp(gmask);
-                const uint32_t src = ring_s + cur * CELLB;
-#pragma unroll
-                for (int c = 0; c < NC; ++c) {
-                    float4 a;
-                    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];\n" : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w) : "r"(src + c * LPT * 16) : "memory");
-                    k0[4 * c] = a.x; k0[4 * c + 1] = a.y; k0[4 * c + 2] = a.z; k0[4 * c + 3] = a.w;
-                    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];\n" : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w) : "r"(src + 512 + c * LPT * 16) : "memory");
-                    v0[4 * c] = a.x; v0[4 * c + 1] = a.y; v0[4 * c + 2] = a.z; v0[4 * c + 3] = a.w;
-                }
-                // and request the cell of the next run (if the run starts inside this group's share)
-                const int pos = (int)((lp - list_s) >> 3);
-                int nxt = -1;
-                for (int base = pos + 1; base < r1 && nxt < 0; base += LPT) {
-                    const int i = base + lg;
-                    const bool f = (i < r1) && (lds_u32(list_s + (uint32_t)i * 8u + 4u) & KVR_CL_FLAG);
-                    const unsigned mm = (__ballot_sync(gmask, f) >> (lane & (32 - LPT))) & ((1u << LPT) - 1u);
-                    if (mm) nxt = base + __ffs(mm) - 1;
-                }
-                cur ^= 1u;
-                if (nxt >= 0) fetch_row0(lds_u32(list_s + (uint32_t)nxt * 8u + 4u) >> KVR_CL_C0_SHIFT, cur);
-            }
-            const uint32_t a1 = lane_cells + (e.x & 0xFFFFu) * CELLB, a2 = lane_cells + (e.x >> 16) * CELLB;
-            // med(g0 a, g1 b, g2 c) = g0 med(a, g0 g1 b, g0 g2 c): g0 folds into the softmax weight
-            const float4 sg = *reinterpret_cast<const float4*>(reinterpret_cast<const char*>(s_sign) + (e.y & 0x70u));
-            const u64 g01p = pack2(sg.y, sg.y), g02p = pack2(sg.z, sg.z);
-            wsign = MEAN ? sg.x * (1.0f / 3.0f) : sg.x;
-            static_for<0, NC>([&](auto ic) {
-                constexpr int c = decltype(ic)::value;
-                const float4 kb = lds_cell<c * LPT * 16>(a1), kc = lds_cell<c * LPT * 16>(a2);
-                if constexpr (MEAN) {
-                    const u64 third2 = pack2(1.0f / 3.0f, 1.0f / 3.0f);
-                    kp[2 * c] = mul2(add2(pack2(kc.x, kc.y), add2(pack2(kb.x, kb.y), pack2(k0[4 * c], k0[4 * c + 1]))), third2);
-                    kp[2 * c + 1] = mul2(add2(pack2(kc.z, kc.w), add2(pack2(kb.z, kb.w), pack2(k0[4 * c + 2], k0[4 * c + 3]))), third2);
-                } else {
-                    kp[2 * c] = pack2(kvr_med3(k0[4 * c], kb.x, kc.x), kvr_med3(k0[4 * c + 1], kb.y, kc.y));
-                    kp[2 * c + 1] = pack2(kvr_med3(k0[4 * c + 2], kb.z, kc.z), kvr_med3(k0[4 * c + 3], kb.w, kc.w));
-                }
-            });
-            static_for<0, NC>([&](auto ic) {
-                constexpr int c = decltype(ic)::value;
-                const float4 vb = lds_cell<512 + c * LPT * 16>(a1), vc = lds_cell<512 + c * LPT * 16>(a2);
-                if constexpr (MEAN) {
-                    // (the sum of the three; its third goes into the softmax weight below)
-                    vp[2 * c] = fma2(pack2(vc.x, vc.y), g02p, fma2(pack2(vb.x, vb.y), g01p, pack2(v0[4 * c], v0[4 * c + 1])));
-                    vp[2 * c + 1] = fma2(pack2(vc.z, vc.w), g02p, fma2(pack2(vb.z, vb.w), g01p, pack2(v0[4 * c + 2], v0[4 * c + 3])));
-                    return;
-                }
-                float b0, b1, b2, b3, c0, c1, c2, c3;
-                unpack2(mul2(pack2(vb.x, vb.y), g01p), b0, b1);
-                unpack2(mul2(pack2(vb.z, vb.w), g01p), b2, b3);
-                unpack2(mul2(pack2(vc.x, vc.y), g02p), c0, c1);
-                unpack2(mul2(pack2(vc.z, vc.w), g02p), c2, c3);
-                vp[2 * c] = pack2(kvr_med3(v0[4 * c], b0, c0), kvr_med3(v0[4 * c + 1], b1, c1));
-                vp[2 * c + 1] = pack2(kvr_med3(v0[4 * c + 2], b2, c2), kvr_med3(v0[4 * c + 3], b3, c3));
-            });
-        };
-        uint32_t lp = list_s + (uint32_t)r0 * 8u;
-        u64 kp[NP], vp[NP];
-        float wsign;
-        if (qn > 0) {
-            reconstruct(lp, true, true, kp, vp, wsign);
-            accumulate(kp, vp, wsign, true);
-            lp += 8;
+            for (int x = 0; x < DPL; ++x) k0[x] = 0.f;
+            const uint32_t own4 = (uint32_t)(own * 4);
+            auto key_token = [&](uint32_t dp, bool live) {
+                uint4 d;
+                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(d.x), "=r"(d.y), "=r"(d.z), "=r"(d.w) : "r"(dp) : "memory");
+                if (live && (d.w & KVR_CL_FLAG)) switch_run(k0, g0K, d.w >> KVR_CL_NEXT_SHIFT);
+                const uint32_t a1 = d.x + lane16, a2 = d.y + lane16;
+                u64 kp[NP];
+                static_for<0, NC>([&](auto ic) {
+                    constexpr int c = decltype(ic)::value;
+                    const float4 kb = lds_cell<c * LPT * 16>(a1), kc = lds_cell<c * LPT * 16>(a2);
+                    if constexpr (MEAN) {
+                        const u64 third2 = pack2(1.0f / 3.0f, 1.0f / 3.0f);
+                        kp[2 * c] = mul2(add2(pack2(kc.x, kc.y), add2(pack2(kb.x, kb.y), pack2(k0[4 * c], k0[4 * c + 1]))), third2);
+                        kp[2 * c + 1] = mul2(add2(pack2(kc.z, kc.w), add2(pack2(kb.z, kb.w), pack2(k0[4 * c + 2], k0[4 * c + 3]))), third2);
+                    } else {
+                        kp[2 * c] = pack2(kvr_med3(k0[4 * c], kb.x, kc.x), kvr_med3(k0[4 * c + 1], kb.y, kc.y));
+                        kp[2 * c + 1] = pack2(kvr_med3(k0[4 * c + 2], kb.z, kc.z), kvr_med3(k0[4 * c + 3], kb.w, kc.w));
+                    }
+                });
+                const float mine = logit(kp);
+                if (live) sts_f32(d.z + own4, mine);
+            };
+            uint32_t dp = desc_s + (uint32_t)r0 * 16u;
 #pragma unroll 1
-            for (int it = 1; it < qn; ++it, lp += 8) {
-                reconstruct(lp, true, false, kp, vp, wsign);
-                accumulate(kp, vp, wsign, true);
+            for (int it = 0; it < qn; ++it, dp += 16) key_token(dp, true);
+            if (rn > 0) key_token(ragged_live ? dp : desc_s, ragged_live);      // ragged last round
+            // the value half of the first token's row-0 cell, for the value pass
+            asm volatile("cp.async.wait_all;\n" ::: "memory");
+            if (qn + (ragged_live ? 1 : 0) > 0) fetch_row0(g0K + (size_t)KVR_R * b * KVR_D, c0_first, 0u);
+        }
+        __syncthreads();
+        // ------------------------------------------------------------ logits -> weights, in place: the
+        // CTA's maximum per head, then w = 2^(logit - max) (times g_0 for a reconstructed token), and
+        // the sums.  NT is a multiple of G: a thread stays with one head.
+        {
+            const int n_tok = nrows + len;
+            float* w = reinterpret_cast<float*>(smem + L.wbuf);
+            auto load_tok = [&](int t, float (&x)[G]) {
+                if constexpr (G == 4) { const float4 v = *reinterpret_cast<const float4*>(w + 4 * t); x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w; }
+                else if constexpr (G == 2) { const float2 v = *reinterpret_cast<const float2*>(w + 2 * t); x[0] = v.x; x[1] = v.y; }
+                else x[0] = w[t];
+            };
+            float mx[G];
+#pragma unroll
+            for (int g = 0; g < G; ++g) mx[g] = M_EMPTY;
+            for (int t = tid; t < n_tok; t += NT) {
+                float x[G];
+                load_tok(t, x);
+#pragma unroll
+                for (int g = 0; g < G; ++g) mx[g] = fmaxf(mx[g], x[g]);
+            }
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+#pragma unroll
+                for (int x = 1; x < 32; x <<= 1) mx[g] = fmaxf(mx[g], __shfl_xor_sync(FULL, mx[g], x));
+                if (lane == 0) s_red[warp][g] = mx[g];
+            }
+            __syncthreads();
+            if (warp == 0) {
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    float v = lane < NW ? s_red[lane][g] : M_EMPTY;
+#pragma unroll
+                    for (int x = 1; x < 32; x <<= 1) v = fmaxf(v, __shfl_xor_sync(FULL, v, x));
+                    if (lane == 0) s_M[g] = v;
+                }
+            }
+            __syncthreads();
+            float M[G], l[G];
+#pragma unroll
+            for (int g = 0; g < G; ++g) { M[g] = s_M[g]; l[g] = 0.f; }
+            for (int t = tid; t < n_tok; t += NT) {
+                float x[G];
+                load_tok(t, x);
+                float sgn = 1.f;
+                if (t >= nrows) {
+                    if (lds_u32(desc_s + (uint32_t)(t - nrows) * 16u + 12u) & (1u << KVR_CL_SIGN_SHIFT)) sgn = -1.f;   // g_0
+                    if (MEAN) sgn *= (1.0f / 3.0f);
+                }
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    const float pr = ex2(x[g] - M[g]);
+                    l[g] += pr;
+                    x[g] = pr * sgn;
+                }
+                if constexpr (G == 4) *reinterpret_cast<float4*>(w + 4 * t) = make_float4(x[0], x[1], x[2], x[3]);
+                else if constexpr (G == 2) *reinterpret_cast<float2*>(w + 2 * t) = make_float2(x[0], x[1]);
+                else w[t] = x[0];
+            }
+            if (tid < G) w[(extra ? p.rcap_extra : p.rcap + lcap) * G + tid] = 0.f;    // the weight of a filler token
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+#pragma unroll
+                for (int x = 1; x < 32; x <<= 1) l[g] += __shfl_xor_sync(FULL, l[g], x);
+                if (lane == 0) s_red[warp][g] = l[g];     // (the maxima in s_red were consumed before the barrier above)
+            }
+            __syncthreads();
+            if (warp == 0) {
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    float v = lane < NW ? s_red[lane][g] : 0.f;
+#pragma unroll
+                    for (int x = 1; x < 32; x <<= 1) v += __shfl_xor_sync(FULL, v, x);      // a fixed tree: same sum every run
+                    if (lane == 0) s_L[g] = v;
+                }
             }
         }
-        if (rn > 0) {                                          // ragged last round
-            const bool live = grp < rn;
-            reconstruct(live ? lp : list_s, live, qn == 0, kp, vp, wsign);
-            accumulate(kp, vp, wsign, live);
-        }
-    }
-
-    // ---------------------------------------------------------------- merge the groups of this CTA
-    __syncthreads();        // ring slots are free: they become the scratch of the merge below
-    {
-        float o[G][DPL];
+        // ------------------------------------------------------------ value pass
+        u64 o2[G][NP];
 #pragma unroll
         for (int g = 0; g < G; ++g)
 #pragma unroll
-            for (int k = 0; k < NP; ++k) unpack2(o2[g][k], o[g][2 * k], o[g][2 * k + 1]);
-        float m_all[G];
-#pragma unroll
-        for (int g = 0; g < G; ++g) m_all[g] = __shfl_sync(FULL, m_own, g << SH, LPT);
-        auto own_of = [&](const float (&v)[G]) {      // v[own] without indexing registers dynamically
-            float r = v[0];
-#pragma unroll
-            for (int g = 1; g < G; ++g) r = (g == own) ? v[g] : r;
-            return r;
-        };
-        // the groups of a warp
-#pragma unroll
-        for (int off = LPT; off < 32; off <<= 1) {
-            float cs_own = 1.f, co_own = 0.f;
-#pragma unroll
-            for (int g = 0; g < G; ++g) {
-                const float mo = __shfl_xor_sync(FULL, m_all[g], off);
-                const float M = fmaxf(m_all[g], mo);
-                const float cs = ex2(m_all[g] - M), co = ex2(mo - M);
-#pragma unroll
-                for (int xx = 0; xx < DPL; ++xx) o[g][xx] = o[g][xx] * cs + __shfl_xor_sync(FULL, o[g][xx], off) * co;
-                m_all[g] = M;
-                if (g == own) { cs_own = cs; co_own = co; }
+            for (int k = 0; k < NP; ++k) o2[g][k] = 0ull;
+        // o[g] += w[g] * v for the token whose weights sit at shared address wa
+        auto add_token = [&](uint32_t wa, const u64 (&vp)[NP]) {
+            float wg[G];
+            if constexpr (G == 4) {
+                const float4 w4 = lds_vol(wa);
+                wg[0] = w4.x; wg[1] = w4.y; wg[2] = w4.z; wg[3] = w4.w;
+            } else if constexpr (G == 2) {
+                asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];\n" : "=f"(wg[0]), "=f"(wg[1]) : "r"(wa) : "memory");
+            } else {
+                asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(wg[0]) : "r"(wa) : "memory");
             }
-            l_own = l_own * cs_own + __shfl_xor_sync(FULL, l_own, off) * co_own;
-        }
-        // every warp leaves its state in shared memory (a record is o[G][128], then m, l per head:
-        // PART floats per head); then one thread per (head, channel) folds the NW records in a fixed
-        // order and writes the CTA's record
-        float* scr = s_ring;
-        const bool speaks = (lg & ((1 << SH) - 1)) == 0;      // one lane per head writes max and sum
-        if (lane < LPT) {
-            float* r = scr + (size_t)warp * G * PART;
 #pragma unroll
             for (int g = 0; g < G; ++g) {
+                const u64 w2 = pack2(wg[g], wg[g]);
 #pragma unroll
-                for (int c = 0; c < NC; ++c) {
-                    float2* d2 = reinterpret_cast<float2*>(r + g * PART + (c * LPT + lg) * 4);   // PART is even: 8-byte aligned
-                    d2[0] = make_float2(o[g][4 * c], o[g][4 * c + 1]);
-                    d2[1] = make_float2(o[g][4 * c + 2], o[g][4 * c + 3]);
+                for (int k = 0; k < NP; ++k) o2[g][k] = fma2(w2, vp[k], o2[g][k]);
+            }
+        };
+        if (nrows > 0) {
+            const uint2* Vr = p.Vr + ((size_t)u * p.R + rb) * 32 + lg;
+            auto rows_val = [&](auto FLc, auto CHK, int base) {
+                constexpr int FLn = decltype(FLc)::value;
+                constexpr bool CHECK = decltype(CHK)::value;
+                const uint2* vb = Vr + (size_t)(base + grp) * 32;
+                uint2 vx[FLn][NC];
+#pragma unroll
+                for (int i = 0; i < FLn; ++i) {
+                    const bool ok = !CHECK || base + i * NGRP + grp < nrows;
+#pragma unroll
+                    for (int c = 0; c < NC; ++c) vx[i][c] = ld_stream8((ok ? vb + i * NGRP * 32 : Vr) + c * LPT);
+                }
+                const uint32_t wa = wbuf_s + (uint32_t)(base + grp) * (G * 4);
+#pragma unroll
+                for (int i = 0; i < FLn; ++i) {
+                    u64 vp[NP], t2[2];
+#pragma unroll
+                    for (int c = 0; c < NC; ++c) { unpack4<T>(vx[i][c], t2); vp[2 * c] = t2[0]; vp[2 * c + 1] = t2[1]; }
+                    add_token((!CHECK || base + i * NGRP + grp < nrows) ? wa + i * NGRP * G * 4 : wzero_s, vp);
+                }
+            };
+            int base = 0;
+            for (; base + FLB * NGRP <= nrows; base += FLB * NGRP) rows_val(std::integral_constant<int, FLB>{}, std::false_type{}, base);
+            for (; base < nrows; base += FLT * NGRP) rows_val(std::integral_constant<int, FLT>{}, std::true_type{}, base);
+        }
+        if (len > 0) {
+            float v0[DPL];
+#pragma unroll
+            for (int x = 0; x < DPL; ++x) v0[x] = 0.f;
+            const float* g0V = g0K + (size_t)KVR_R * b * KVR_D;
+            auto val_token = [&](uint32_t dp, bool live) {
+                uint4 d;
+                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(d.x), "=r"(d.y), "=r"(d.z), "=r"(d.w) : "r"(dp) : "memory");
+                if (live && (d.w & KVR_CL_FLAG)) switch_run(v0, g0V, d.w >> KVR_CL_NEXT_SHIFT);
+                const uint32_t a1 = d.x + lane16, a2 = d.y + lane16;
+                // med(g0 a, g1 b, g2 c) = g0 med(a, g0 g1 b, g0 g2 c): g0 is part of the weight
+                const float4 sg = lds_vol(d.w & 0xFFF0u);
+                const u64 g01p = pack2(sg.x, sg.y), g02p = pack2(sg.z, sg.w);
+                u64 vp[NP];
+                static_for<0, NC>([&](auto ic) {
+                    constexpr int c = decltype(ic)::value;
+                    const float4 vb = lds_cell<HALFB + c * LPT * 16>(a1), vc = lds_cell<HALFB + c * LPT * 16>(a2);
+                    if constexpr (MEAN) {
+                        // (the sum of the three; its third is part of the weight)
+                        vp[2 * c] = fma2(pack2(vc.x, vc.y), g02p, fma2(pack2(vb.x, vb.y), g01p, pack2(v0[4 * c], v0[4 * c + 1])));
+                        vp[2 * c + 1] = fma2(pack2(vc.z, vc.w), g02p, fma2(pack2(vb.z, vb.w), g01p, pack2(v0[4 * c + 2], v0[4 * c + 3])));
+                        return;
+                    }
+                    float b0, b1, b2, b3, c0, c1, c2, c3;
+                    unpack2(mul2(pack2(vb.x, vb.y), g01p), b0, b1);
+                    unpack2(mul2(pack2(vb.z, vb.w), g01p), b2, b3);
+                    unpack2(mul2(pack2(vc.x, vc.y), g02p), c0, c1);
+                    unpack2(mul2(pack2(vc.z, vc.w), g02p), c2, c3);
+                    vp[2 * c] = pack2(kvr_med3(v0[4 * c], b0, c0), kvr_med3(v0[4 * c + 1], b1, c1));
+                    vp[2 * c + 1] = pack2(kvr_med3(v0[4 * c + 2], b2, c2), kvr_med3(v0[4 * c + 3], b3, c3));
+                });
+                add_token(live ? d.z : wzero_s, vp);
+            };
+            uint32_t dp = desc_s + (uint32_t)r0 * 16u;
+#pragma unroll 1
+            for (int it = 0; it < qn; ++it, dp += 16) val_token(dp, true);
+            if (rn > 0) val_token(ragged_live ? dp : desc_s, ragged_live);
+        }
+        // ------------------------------------------------------------ add up the groups of this CTA (they
+        // share one maximum, so this is a plain sum in a fixed order) and fold the stretch into the record
+        asm volatile("cp.async.wait_all;\n" ::: "memory");         // no copy into the ring is in flight
+        {
+            // every group leaves its sums in shared memory, as many groups at a time as fit between
+            // the ring and the cells (descriptors and weights are no longer needed); one thread per
+            // (head, channel) adds them in group order
+            float* scr = reinterpret_cast<float*>(smem + L.ring);   // [groups at a time][G][128]
+            const int fit = min(NGRP, (L.cells - L.ring) / (G * HALFB));
+            float sum = 0.f;
+            for (int g0 = 0; g0 < NGRP; g0 += fit) {
+                __syncthreads();
+                if (grp >= g0 && grp < g0 + fit) {
+                    float* r = scr + (size_t)(grp - g0) * G * KVR_D;
+#pragma unroll
+                    for (int g = 0; g < G; ++g)
+#pragma unroll
+                        for (int c = 0; c < NC; ++c) {
+                            float4 v;
+                            unpack2(o2[g][2 * c], v.x, v.y);
+                            unpack2(o2[g][2 * c + 1], v.z, v.w);
+                            *reinterpret_cast<float4*>(r + g * KVR_D + (c * LPT + lg) * 4) = v;
+                        }
+                }
+                __syncthreads();
+                if (tid < G * KVR_D) {
+                    const int n = min(fit, NGRP - g0);
+#pragma unroll 4
+                    for (int w = 0; w < n; ++w) sum += scr[w * G * KVR_D + tid];
                 }
             }
-            if (speaks) { r[own * PART + KVR_D] = own_of(m_all); r[own * PART + KVR_D + 1] = l_own; }
-        }
-        __syncthreads();
-    }
-    // Block coordinates are read again here rather than kept in registers through the token loop,
-    // where every register counts.
-    uint32_t bx, by, nbx, tx;
-    asm volatile("mov.u32 %0, %%ctaid.x;\n mov.u32 %1, %%ctaid.y;\n mov.u32 %2, %%nctaid.x;\n mov.u32 %3, %%tid.x;\n"
-                 : "=r"(bx), "=r"(by), "=r"(nbx), "=r"(tx));
-    {
-        const float* scr = s_ring;
-        float* part = p.part + ((size_t)by * nbx + bx) * G * PART;
-        for (int idx = (int)tx; idx < G * KVR_D; idx += NT) {
-            const int g = idx >> 7, d = idx & (KVR_D - 1);
-            float M = M_EMPTY;
-#pragma unroll
-            for (int w = 0; w < NW; ++w) M = fmaxf(M, scr[(w * G + g) * PART + KVR_D]);
-            float Lsum = 0.f, O = 0.f;
-#pragma unroll
-            for (int w = 0; w < NW; ++w) {
-                const float f = ex2(scr[(w * G + g) * PART + KVR_D] - M);
-                Lsum += scr[(w * G + g) * PART + KVR_D + 1] * f;
-                O += scr[(w * G + g) * PART + d] * f;
+            const int g = tid >> 7, d = tid & (KVR_D - 1);
+            float Mo = M_EMPTY, Lo = 0.f, Oo = 0.f;
+            if (st > 0 && tid < G * KVR_D) { Mo = s_acc[g * PART + KVR_D]; Lo = s_acc[g * PART + KVR_D + 1]; Oo = s_acc[g * PART + d]; }
+            if (st > 0) __syncthreads();
+            if (tid < G * KVR_D) {
+                const float Ms = s_M[g], Mn = fmaxf(Mo, Ms);
+                const float f0 = ex2(Mo - Mn), f1 = ex2(Ms - Mn);
+                s_acc[g * PART + d] = Oo * f0 + sum * f1;
+                if (d == 0) { s_acc[g * PART + KVR_D] = Mn; s_acc[g * PART + KVR_D + 1] = Lo * f0 + s_L[g] * f1; }
             }
-            part[g * PART + d] = O;
-            if (d == 0) { part[g * PART + KVR_D] = M; part[g * PART + KVR_D + 1] = Lsum; }
         }
     }
-    finish_instance<G, NT>(p.part + (size_t)by * nbx * G * PART, (int)nbx, &p.tickets[p.inst0 + by],
-                           p.out + (size_t)by * G * KVR_D, p.ml + (size_t)(p.inst0 + by) * G * 2,
-                           reinterpret_cast<int*>(smem + make_layout(p.n1, p.lcap).flag));
+    // ---------------------------------------------------------------- everything above reads only what no
+    // decode launch writes (cells, token lists, the caller's rows and queries) and writes shared
+    // memory only.  When this launch was made a programmatic dependent of the previous decode launch,
+    // its CTAs took over the SMs that launch freed one by one and may have run beside its last CTAs:
+    // wait for that launch to be complete here, before the first write to global memory (records,
+    // tickets, outputs are shared by consecutive launches).
+    asm volatile("griddepcontrol.wait;\n" ::: "memory");
+    __syncthreads();
+    {
+        float* part = p.part + ((size_t)blockIdx.y * gridDim.x + blockIdx.x) * G * PART;
+        for (int i = tid; i < G * PART; i += NT) part[i] = s_acc[i];
+    }
+    finish_instance<G, NT>(p.part + (size_t)blockIdx.y * gridDim.x * G * PART, (int)gridDim.x, &p.tickets[p.inst0 + blockIdx.y],
+                           p.out + (size_t)blockIdx.y * G * KVR_D, p.ml + (size_t)(p.inst0 + blockIdx.y) * G * 2,
+                           reinterpret_cast<int*>(smem + L.ctrl));
 }
 
 // chained: the previous kernel of the stream is a staged decode launch of the same handle and nothing
 // has changed the handle's cells or lists since, so this launch may overlap its start with that
 // launch's end (programmatic dependent launch; the kernel waits before it touches anything shared).
-template <typename T, int G, int LPT, bool MEAN>
+template <typename T, int G, bool MEAN>
 cudaError_t launch_one(const StagedParams& p, int n_inst, int grid_x, size_t smem, bool chained, cudaStream_t st) {
-    auto kern = decode_staged_kernel<T, G, LPT, MEAN>;
+    auto kern = decode_staged_kernel<T, G, MEAN>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid_x, n_inst);
-    cfg.blockDim = dim3(NGRP * LPT);
+    cfg.blockDim = dim3(NT);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -629,36 +762,29 @@ cudaError_t launch_one(const StagedParams& p, int n_inst, int grid_x, size_t sme
 }  // namespace
 
 // Smallest class grid whose rows-1-and-2 slices leave room for the ring and a useful number of
-// token entries; 0 when the sketch is too wide (or the query group too large) for this kernel.
+// token entries and logits; 0 when the sketch is too wide (or the query group too large) for this kernel.
 int kvr_decode_staged_pick_C(int b, int G) {
     if (G != 1 && G != 2 && G != 4) return 0;
     for (int C = 1; C <= 8; C *= 2) {
         const int n1 = (b + C - 1) / C;
-        if ((size_t)make_layout(n1, 1024).total <= SMEM_LIMIT) return C;
+        if (2 * n1 <= 226 && (size_t)make_layout(n1, 1536, 768, G).total <= SMEM_LIMIT) return C;
     }
     return 0;
 }
 
 // How the staged kernel would run this call, or `false` when it cannot (no class grid fits) or
-// should not (so few tokens that almost every one would fetch its own row-0 cell from global memory;
-// measured: at one token per class and row-0 cell the staged kernel is still 1.6x faster than the split one).
+// should not (so few tokens that almost every one would fetch its own row-0 cell from global memory).
 bool kvr_decode_staged_plan(const kvr_sketch* sk, int n_inst, int N, int R, int rows, bool forced,
                             KvrStagedPlan* plan) {
-    const int a = N - R, C = sk->C;
+    const int a = N - R, C = sk->C, G = sk->G;
     R = rows;                                   // from here on: the rows to stream
     if (C < 1 || a < 1) return false;
     const int n_cls = C * C;
     if (!forced && 2LL * a < (long long)sk->d.b * n_cls) return false;   // under half a token per (class, row-0 cell)
-    int S = sk->n_sm / (n_inst * n_cls);                      // one CTA per SM (the kernel fills the register file)
+    int S = sk->n_sm / (n_inst * n_cls);                      // one CTA per SM
     if (S < 1) S = 1;
-    const int s_cap = a / (n_cls * 2 * NGRP) > 0 ? a / (n_cls * 2 * NGRP) : 1;   // a couple of tokens per half-warp at least
+    const int s_cap = a / (n_cls * 2 * NGRP) > 0 ? a / (n_cls * 2 * NGRP) : 1;   // a couple of tokens per group at least
     if (S > s_cap) S = s_cap;
-    // entries staged at a time: the expected slice with head-room, bounded by what shared memory leaves
-    long long want = (long long)a / (n_cls * S);
-    want += want / 4 + 64;
-    const long long room = ((long long)SMEM_LIMIT - make_layout(sk->n1, 0).total) / 8 - 2;
-    if (want > room) want = room;
-    if (want > a) want = a;
     // SMs the class CTAs leave idle stream retained rows only.  The rows are dealt so that all CTAs
     // finish at about the same time.
     const int n_ccta = n_cls * S;
@@ -674,12 +800,33 @@ bool kvr_decode_staged_plan(const kvr_sketch* sk, int n_inst, int N, int R, int 
         r_cls = (int)(x * n_ccta);
         if (r_cls >= R) { r_cls = R; extra = 0; }
     }
+    // entries and rows kept on chip at a time: the expected slice with head-room, and the class CTA's
+    // rows, both cut down together when shared memory does not hold them (the kernel then takes its
+    // tokens in several stretches)
+    long long want_l = (long long)a / n_ccta;
+    want_l += want_l / 8 + 64;
+    if (want_l > a) want_l = a;
+    long long want_r = (r_cls + n_ccta - 1) / n_ccta + 1;
+    const long long room = (long long)SMEM_LIMIT - make_layout(sk->n1, 0, 0, G).total - 128;
+    const long long need = want_l * (16 + 4 * G) + want_r * 4 * G;     // descriptor + logits per entry, logits per row
+    bool cut = false;
+    if (need > room) {
+        want_l = want_l * room / need;
+        want_r = want_r * room / need;
+        if (want_l < 2) want_l = 2;
+        if (want_r < 1) want_r = 1;
+        cut = true;
+    }
+    want_l = cut ? (want_l & ~1LL) : ((want_l + 1) & ~1LL);       // an even number of entries
     plan->S = S;
-    plan->lcap = (int)want;
+    plan->lcap = (int)want_l;
+    plan->rcap = (int)want_r;
     plan->extra = extra;
     plan->r_cls = r_cls;
     plan->records = n_ccta + extra;
-    plan->smem = (size_t)make_layout(sk->n1, plan->lcap).total;
+    const Layout L = make_layout(sk->n1, plan->lcap, plan->rcap, G);
+    plan->smem = (size_t)L.total;
+    plan->rcap_extra = (L.total - L.wbuf) / (4 * G) - 1;      // a row-only CTA keeps logits where the others keep entries and cells
     return true;
 }
 
@@ -709,8 +856,11 @@ cudaError_t kvr_launch_decode_staged(kvr_sketch* sk, int inst0, int n_inst, int 
     p.max_ctx = sk->d.max_context;
     p.S = plan.S;
     p.lcap = plan.lcap;
+    p.rcap = plan.rcap;
+    p.rcap_extra = plan.rcap_extra;
     p.n_ccta = plan.records - plan.extra;
     p.r_cls = plan.r_cls;
+    p.zero = 0u;
     p.scale_log2e = scale * 1.4426950408889634f;
     sk->launches += 1;
     const bool f16 = sk->d.kv_dtype == KVR_F16;
@@ -718,12 +868,12 @@ cudaError_t kvr_launch_decode_staged(kvr_sketch* sk, int inst0, int n_inst, int 
     const bool chained = sk->chain && sk->chain_stream == st;
     sk->chain = true;
     sk->chain_stream = st;
-#define KVR_STAGED(GG)                                                                                              \
-    case GG:                                                                                                        \
-        if (sk->combine) return f16 ? launch_one<__half, GG, KVR_LPT, true>(p, n_inst, gx, plan.smem, chained, st)  \
-                                    : launch_one<__nv_bfloat16, GG, KVR_LPT, true>(p, n_inst, gx, plan.smem, chained, st); \
-        return f16 ? launch_one<__half, GG, KVR_LPT, false>(p, n_inst, gx, plan.smem, chained, st)                  \
-                   : launch_one<__nv_bfloat16, GG, KVR_LPT, false>(p, n_inst, gx, plan.smem, chained, st);
+#define KVR_STAGED(GG)                                                                                     \
+    case GG:                                                                                               \
+        if (sk->combine) return f16 ? launch_one<__half, GG, true>(p, n_inst, gx, plan.smem, chained, st)  \
+                                    : launch_one<__nv_bfloat16, GG, true>(p, n_inst, gx, plan.smem, chained, st); \
+        return f16 ? launch_one<__half, GG, false>(p, n_inst, gx, plan.smem, chained, st)                  \
+                   : launch_one<__nv_bfloat16, GG, false>(p, n_inst, gx, plan.smem, chained, st);
     switch (sk->G) {
         KVR_STAGED(1)
         KVR_STAGED(2)

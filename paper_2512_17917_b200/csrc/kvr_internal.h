@@ -22,14 +22,17 @@
 #define KVR_PACK_H_MASK 0x1FFFu
 
 // Per compressed token, for the staged decode kernel (tokens grouped by class, see kvr_sketch::C):
-//   x: bits 0-15 = index of the row-1 cell inside the class's slice, bits 16-31 = index of the
-//      row-2 cell inside the staged array (row-2 slice follows the row-1 slice)
+//   x: bits 0-7 = index of the row-1 cell inside the class's slice, bits 8-15 = index of the row-2
+//      cell inside the staged array (row-2 slice follows the row-1 slice; the array has at most 226
+//      cells of 1 KB), bits 16-31 = row-0 cell of the next flagged entry of the list (the cell
+//      the kernel fetches ahead while it works on this entry's run)
 //   y: bit 0 = first token of its row-0 cell inside its class (the row-0 cell must be reloaded),
 //      bit 4 = g_0 is -1, bit 5 = g_0 g_1 is -1, bit 6 = g_0 g_2 is -1 (so that y & 0x70 is the byte
-//      offset of a 16-byte row in a table of sign triples), bits 16-31 = row-0 cell
+//      offset of a 16-byte row in a table of sign pairs), bits 16-31 = row-0 cell
 #define KVR_CL_FLAG 1u
 #define KVR_CL_SIGN_SHIFT 4
 #define KVR_CL_C0_SHIFT 16
+#define KVR_CL_NEXT_SHIFT 16
 
 struct kvr_sketch {
     kvr_sketch_desc_t d;
@@ -100,6 +103,8 @@ struct kvr_sketch {
 struct KvrStagedPlan {
     int S;         // token slices per class
     int lcap;      // token entries staged at a time
+    int rcap;      // retained rows of a class CTA whose logits are kept on chip at a time
+    int rcap_extra;  // the same for a CTA that only streams rows
     int extra;     // CTAs per head-instance that only stream retained rows (SMs the classes leave idle)
     int r_cls;     // retained rows handled by the class CTAs (the rest go to the extra CTAs)
     int records;   // partial records per head-instance (C*C*S + extra)

@@ -111,7 +111,8 @@ __global__ void csr_fill_kernel(const int32_t* __restrict__ tok_h, const int32_t
 //                  row-0-cell order, ascending token index inside a cell, as packed entries
 //   clist / coff   (when the handle has a class grid, C > 0) the same tokens regrouped into C x C
 //                  classes by (row-1 cell mod C, row-2 cell mod C), row-0-cell order kept inside each
-//                  class, the first token of every row-0 cell inside its class flagged
+//                  class, the first token of every row-0 cell inside its class flagged and told the
+//                  row-0 cell of the run that follows it
 // One cluster of LST_CL CTAs per head-instance; CTA r owns a contiguous range of row-0 cells, one
 // warp a cell at a time.  Pass 1 counts the kept tokens per (cell, class); the CTAs exchange their
 // column sums through distributed shared memory (cluster barriers, nothing spins); ordered scans turn
@@ -255,7 +256,7 @@ lists_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ f
                     const uint32_t h1 = e & KVR_PACK_H_MASK, h2 = (e >> KVR_PACK_H2_SHIFT) & KVR_PACK_H_MASK;
                     const uint32_t sg = e >> KVR_PACK_SIGN_SHIFT;
                     const uint32_t s3 = (sg & 1u) | (((sg ^ (sg >> 1)) & 1u) << 1) | (((sg ^ (sg >> 2)) & 1u) << 2);
-                    cl[row[1 + k] + seen] = make_uint2((h1 >> logC) | (((uint32_t)n1 + (h2 >> logC)) << 16),
+                    cl[row[1 + k] + seen] = make_uint2((h1 >> logC) | (((uint32_t)n1 + (h2 >> logC)) << 8),
                                                        ((uint32_t)c << KVR_CL_C0_SHIFT) | (s3 << KVR_CL_SIGN_SHIFT) |
                                                            (seen == 0 ? KVR_CL_FLAG : 0u));
                 }
@@ -265,7 +266,23 @@ lists_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ f
             }
         }
     }
-    cluster.sync();                      // no CTA leaves while another may still read its column sums
+    cluster.sync();                      // no CTA leaves while another may still read its column sums;
+                                         // every entry of the class list is written and visible
+    // ---- pass 3: every entry learns the row-0 cell of the next flagged entry of the list (flagged =
+    // first token of a row-0 cell inside its class), which is the cell the decode kernel fetches ahead
+    // while it works on the entry's run.  The first entry of every class is flagged, so a walk ends at
+    // the next class's first entry at the latest; the last run of the list names its own cell.
+    if (n_cls) {
+        const int a = s_all[0];
+        for (int i = crank * LST_THREADS + tid; i < a; i += LST_CL * LST_THREADS) {
+            const uint2 e = cl[i];
+            if (!(e.y & KVR_CL_FLAG)) continue;
+            int j = i + 1;
+            while (j < a && !(cl[j].y & KVR_CL_FLAG)) ++j;
+            const uint32_t nxt = ((j < a ? cl[j].y : e.y) >> KVR_CL_C0_SHIFT) << KVR_CL_NEXT_SHIFT;
+            for (int k = i; k < j; ++k) cl[k].x = (cl[k].x & 0xFFFFu) | nxt;
+        }
+    }
 }
 
 __global__ void assignment_kernel(const int32_t* __restrict__ cmp_all, const int32_t* __restrict__ tok_h,
