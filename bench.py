@@ -101,6 +101,24 @@ class ClockSampler:
         return out
 
 
+def config_of(w) -> dict:
+    """The workload as both arms print it (same keys, so that the two lines can be matched)."""
+    return {"workload": w.name, "batch": w.batch, "layers": w.n_layers, "kv_heads": w.n_kv_heads,
+            "q_heads": w.n_q_heads, "head_dim": w.head_dim, "context": w.context, "budget": w.budget,
+            "sketch_rows": 3, "sketch_width": w.b, "obs_window": w.obs_window,
+            "decode_steps_per_step": w.decode_steps, "kv_dtype": w.dtype, "launch": "per_layer_cuda_graph",
+            "l2": "inputs larger than L2 (each decode step streams %.2f GB)"
+                  % (decode_bytes_per_launch(w, w.n_layers * w.batch * w.n_kv_heads) / 1e9)}
+
+
+def host_cores() -> int:
+    """Cores this process may run on (the oracle's OpenMP team is sized from the same mask)."""
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
 def decode_bytes_per_launch(w, n_inst_launch: int, entry_bytes: int = 8) -> int:
     """Algorithmic HBM bytes of one decode-attention launch over n_inst head-instances: retained
     K and V rows, the fp32 sketch (keys + values) once, the list of compressed tokens (8-byte
@@ -116,6 +134,12 @@ def compress_bytes_per_layer(w, n_inst_layer: int) -> int:
     insertion share them through L2), the retained copies written, the fp32 sketch written."""
     R, N, b, D = w.budget, w.context, w.b, w.head_dim
     return (N * D * 2 * 2 + R * D * 2 * 2 + 3 * b * 2 * D * 4) * n_inst_layer
+
+
+def smem_cell_bytes_per_launch(w, n_inst_launch: int) -> int:
+    """Shared-memory bytes of cell data one staged launch reads: every reconstructed token takes two
+    of its three cells (keys and values, fp32) from shared memory; the third sits in registers."""
+    return (w.context - w.budget) * 2 * 2 * w.head_dim * 4 * n_inst_launch
 
 
 def minmax_ops_per_launch(w, n_inst_launch: int) -> int:
@@ -226,15 +250,28 @@ def run_gpu(args, w, rank, world, local):
                 "frac_of_nominal_8TBs": round(ach / 8000.0, 4),
                 "bytes_per_launch": bytes_launch, "avg_launch_us": round(launch_ms * 1e3, 2),
                 "traffic": args.traffic}
-    # The same launch against the pipe that actually limits it: fp32 min/max issue on the ALU pipe
-    # (64 lanes per clock per SM), the medians of the reconstruction being the unavoidable part.
-    props = torch.cuda.get_device_properties(dev)
-    alu_peak = props.multi_processor_count * 64 * 1.965e9 / 1e12          # T lane-ops/s at the maximum SM clock
+    # The same launch against the two on-chip rates Algorithm 2 cannot avoid, both MEASURED on this
+    # device a moment ago by the library's probe kernels (a register-only min/max loop and a
+    # conflict-free 16-byte shared-memory load loop): the medians run on the ALU pipe, the two cells a
+    # token does not keep in registers are read from shared memory once per pass.
+    mm_peak, lds_peak = kvr.kvr_measure_pipe_peaks()
+    alu_peak = mm_peak / 1e12                                              # T lane-ops/s
     alu_ach = minmax_ops_per_launch(w, B * H) / (launch_ms * 1e-3) / 1e12
     roofline_alu = {"kernel": kernel_name, "bound": "alu", "achieved": round(alu_ach, 3), "peak": round(alu_peak, 3),
                     "unit": "T min/max lane-ops/s", "frac": round(alu_ach / alu_peak, 4),
-                    "peak_kind": "derived: SMs x 64 ALU lanes x 1965 MHz"}
-
+                    "peak_kind": "measured: register-only min/max loop (kvr_measure_pipe_peaks)"}
+    smem_bytes = smem_cell_bytes_per_launch(w, B * H)
+    smem_ach = smem_bytes / (launch_ms * 1e-3) / 1e9
+    roofline_smem = {"kernel": kernel_name, "bound": "smem", "achieved": round(smem_ach, 1),
+                     "peak": round(lds_peak / 1e9, 1), "unit": "GB/s", "frac": round(smem_ach / (lds_peak / 1e9), 4),
+                     "bytes_per_launch": smem_bytes,
+                     "peak_kind": "measured: 16-byte shared-memory load loop (kvr_measure_pipe_peaks)"}
+    # which of the three ceilings is nearest (the largest fraction), and the time each alone would allow
+    floors_us = {"hbm": bytes_launch / (peak * 1e9) * 1e6, "alu": minmax_ops_per_launch(w, B * H) / mm_peak * 1e6,
+                 "smem": smem_bytes / lds_peak * 1e6}
+    binding = {"nearest_ceiling": max(floors_us, key=floors_us.get),
+               "floor_us": {k: round(v, 2) for k, v in floors_us.items()},
+               "note": "the launch also spends instruction issue slots around these; see DESIGN.md section 8"}
     # ---- same decode work as ONE launch over all layers per decode step (upper bound on launch shape) ----
     batched = None
     if L > 1:
@@ -299,10 +336,7 @@ def run_gpu(args, w, rank, world, local):
         "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 3), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": w.name, "batch": B, "layers": L, "kv_heads": H, "q_heads": Hq, "head_dim": D,
-                   "context": N, "budget": R, "sketch_rows": 3, "sketch_width": w.b, "obs_window": W,
-                   "decode_steps_per_step": S, "kv_dtype": w.dtype, "launch": "per_layer_cuda_graph",
-                   "l2": "inputs larger than L2 (each decode step streams %.2f GB)" % (decode_bytes_per_launch(w, L * B * H) / 1e9)},
+        "config": config_of(w),
         "decode_kernel": kernel_name,
         "compress_ms_per_step": round(compress_ms, 3), "decode_ms_per_step": round(decode_ms, 3),
         "compress": {"ms_per_layer": round(compress_ms / L, 4),
@@ -312,7 +346,7 @@ def run_gpu(args, w, rank, world, local):
                      "scoring_kernel": {kvr.KVR_SCORE_TCGEN05: "score_tc_kernel (tcgen05)",
                                         kvr.KVR_SCORE_MMA_SYNC: "score_pass_kernel (mma.sync)"}.get(kvr.kvr_last_score_kernel(sk), "?")},
         "decode_only_tokens_per_s": round(world * B * S / (decode_ms * 1e-3), 1),
-        "roofline": roofline, "roofline_alu": roofline_alu, "layer_batched": batched, "e2e": e2e, "gpu_launches": int(gpu_launches),
+        "roofline": roofline, "roofline_alu": roofline_alu, "roofline_smem": roofline_smem, "binding": binding, "layer_batched": batched, "e2e": e2e, "gpu_launches": int(gpu_launches),
         "clocks": clocks, "checksum": checksum,
         "device_bytes": kvr.kvr_sketch_device_bytes(sk),
     }
@@ -359,7 +393,7 @@ def oracle_throughput(w, compress_s, decode_s, n_sample):
 
 def run_reference(args, w):
     """--impl reference: the CPU oracle on the host cores, each step a bounded sample."""
-    cores = os.cpu_count() or 1
+    cores = host_cores()
     n_sample = max(1, min(cores, w.batch * w.n_kv_heads))
     dsteps = 1
     vals, step_ms = [], []
@@ -376,8 +410,7 @@ def run_reference(args, w):
         "impl": "reference", "metric": METRIC, "value": round(v, 4), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(float(np.mean(step_ms)), 1), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "context": w.context, "budget": w.budget, "sketch_width": w.b,
-                   "layers": w.n_layers, "batch": w.batch},
+        "config": config_of(w),
         "cpu_baseline": {"value": round(v, 4), "unit": UNIT, "cores": used, "kind": "oracle", "sample": sample},
         "e2e": {"value": round(v, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -443,7 +476,7 @@ def main():
     result, inputs = run_gpu(args, w, rank, world, local)
     if rank == 0:
         if not args.no_cpu_baseline:
-            cores = os.cpu_count() or 1
+            cores = host_cores()
             cs, ds, used, ns = oracle_sample(w, max(1, min(cores, w.batch * w.n_kv_heads)), 1, inputs, combine=args.combine)
             v, _ = oracle_throughput(w, cs, ds, ns)
             result["cpu_baseline"] = {

@@ -2,9 +2,8 @@
  * kvr.h -- C ABI of libkvr: the data-parallel hot path of KVReviver (reversible KV-cache
  * compression with sketch-based token reconstruction) for NVIDIA B200 (sm_100a).
  *
- * Two operations, applied independently to every head-instance (batch x layer x kv head; the
- * paper deploys the method "independently on each of the attention layers", Algorithm section,
- * Overview):
+ * Two operations, applied independently to every head-instance (batch x layer x kv head; in the
+ * paper every attention layer runs its own copy of the method: Algorithm section, Overview):
  *
  *   compress          score the N context tokens by accumulated attention of an observation
  *                     window, keep the top-budget tokens exactly (Recent + Candidate parts of
@@ -149,12 +148,14 @@ kvr_status_t kvr_decode_attention(kvr_sketch_t* sk, int32_t layer, const void* q
  * allocating routine.  Its scratch (split partials and arrival tickets) is one fixed array of
  * KVR_STATIC_SCRATCH_BYTES in device global memory that belongs to the library image: every GPU
  * that loads libkvr holds it until the process exits.
- *   - Arguments, results and errors as kvr_decode_attention; in addition KVR_ERR_LIMIT when the
+ *   - Arguments, results and errors as kvr_decode_attention (rows appended after the compress
+ *     included; the split kernel serves the call); in addition KVR_ERR_LIMIT when the
  *     call covers more than 4096 head-instances or needs more split-partial space than the array
  *     has (head-instances x splits x (n_q_heads / n_kv_heads) x 520 bytes; one layer of 8 kv
  *     heads at 32k context needs about 0.9 MiB, 256 head-instances in one launch about 1 MiB).
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress, with
- *     that device current); make that first call before any stream capture begins.
+ *     that device current; host threads that make their first calls together are serialised by a
+ *     lock); make that first call before any stream capture begins.
  *   - All calls on a device share the array, which keeps the previous call's contents; the tickets
  *     are cleared on `cuda_stream` before each launch.  Two calls whose kernels can overlap on the
  *     GPU (different streams, or different handles on different streams) race on it: keep every
@@ -207,9 +208,11 @@ kvr_status_t kvr_demote(kvr_sketch_t* sk, int32_t layer, const void* Kr, const v
 kvr_status_t kvr_accumulate_vague_scores(kvr_sketch_t* sk, int32_t layer, const void* q,
                                          float softmax_scale, void* cuda_stream);
 
-/* Swap loop of Algorithm 3, in place on the caller's exact storage of the layer:
- *     while C.Min_Score() * replace_rate < V.Max_Score() (and fewer than max_swaps swaps were made):
- *         tmp <- V.Query(best vague token);  V.Delete(tmp);  V.Insert(worst candidate);  C.Push(tmp)
+/* Swap loop of Algorithm 3, in place on the caller's exact storage of the layer.  As long as the
+ * best-scored token of the Vague part beats the worst-scored Candidate row by more than the factor
+ * replace_rate (and fewer than max_swaps swaps were made), the two change places: the vague token is
+ * queried from the sketch and taken out of it again, the candidate's vectors go into the sketch, and
+ * the queried vectors take the candidate's row.
  * Kr, Vr [batch, n_kv_heads, n_rows, head_dim] (kv_dtype), ret_idx and row_scores [.., n_rows]: the
  * storage as the layer's last kvr_compress / kvr_demote left it (n_rows = its retained count).  The
  * Candidate part is the rows [0, n_rows - n_recent); the newest n_recent rows are never touched.  A

@@ -21,8 +21,8 @@
  * the same precision on both sides.
  *
  * No blocking, fusion or reordering beyond what the algorithms state.  OpenMP appears only in the
- * *_batch drivers, over independent head-instances ("deployed independently on each of the
- * attention layers", Overview section); each head-instance is plain sequential loops.
+ * *_batch drivers, over independent head-instances (every attention layer runs its own copy of
+ * the method: Overview section); each head-instance is plain sequential loops.
  *
  * Parity pins (tests marked "not gpu"): scores against a library softmax column sum and the
  * row-sum invariant; selection against a full sort; hashing against hand-worked values and the
@@ -89,9 +89,9 @@ void kvro_bucket_sign(const uint32_t *seeds, int32_t mix, int32_t r, int32_t b, 
 }
 
 /* ---------------------------------------------------------------------------------------------
- * Importance scores (Overview section: "retain and accumulate the attention scores for each
- * token, which is the result of Softmax(QK^T)"; scale 1/sqrt(d_k) from the attention-score
- * formula).  Q holds the n_rows = G*W observation queries that share this KV head; none of them
+ * Importance scores (Overview section: a token's importance is the attention probability it
+ * receives, Softmax(QK^T), summed over the queries seen; scale 1/sqrt(d_k) from the
+ * attention-score formula).  Q holds the n_rows = G*W observation queries that share this KV head; none of them
  * is masked (they sit after all N context tokens).
  *     S[t][j] = scale * sum_d Q[t][d] K[j][d];  P[t][.] = softmax_j S[t][.];  s[j] = sum_t P[t][j]
  * ------------------------------------------------------------------------------------------- */
@@ -205,7 +205,7 @@ int32_t kvro_select(const float *s, int32_t N, int32_t R, int32_t n_recent, int3
  *     V[i][h_i(J)].key   += T.key
  *     V[i][h_i(J)].value += T.value * g_i(J)          (signs on values only)
  * cells: [r][b][2][D] doubles, slot 0 = key vector, slot 1 = value vector; the caller zeroes
- * them ("initially all tensors are zeros").  K, V: [N][D] rows of the full cache.
+ * them (the Vague Sketch section starts from an all-zero sketch).  K, V: [N][D] rows of the full cache.
  * sign_scale = +1 inserts, -1 removes (V.Delete by linearity; not used on the one-shot path).
  * ------------------------------------------------------------------------------------------- */
 void kvro_insert(double *cells, const uint32_t *seeds, int32_t mix, int32_t r, int32_t b, int32_t D,
@@ -447,8 +447,8 @@ void kvro_decode_c_batch(int32_t n_inst, const float *q /*[n_inst][G][D]*/, int3
 }
 
 /* ---------------------------------------------------------------------------------------------
- * Attention mass every token receives in one decode step (Overview: the method keeps and
- * accumulates "the attention scores for each token, which is the result of Softmax(QK^T)"):
+ * Attention mass every token receives in one decode step (Overview: the attention probabilities
+ * of every computation are kept and added up per token):
  *     mass[j] = sum over the G query heads of  Softmax_j(q_g K^T * scale)
  * over the rebuilt cache of Algorithm 4.  mass: [N].
  * ------------------------------------------------------------------------------------------- */

@@ -239,10 +239,10 @@ def demote(Kr, Vr, ret_idx, row_scores, cells, budget: int, n_recent: int, seeds
 
 def swap(Kr, Vr, ret_idx, row_scores, tok_scores, cells, n_recent: int, replace_rate: float, max_swaps: int,
          seeds, mix: bool = True, round_rows=None):
-    """Swap loop of Algorithm 3 on one storage, step by step as printed:
-
-        while C.Min_Score() * ReplaceRate < V.Max_Score():
-            tmp <- V.Query(V.Max_Score_Index());  V.Delete(tmp);  V.Insert(C.Top_Pop());  C.Push(tmp)
+    """Swap loop of Algorithm 3 on one storage, one exchange at a time in the algorithm's order: while
+    the lowest Candidate score times ReplaceRate is below the highest Vague score, query that vague
+    token, remove it from the sketch, insert the lowest-scored candidate into the sketch, and give the
+    queried vectors the candidate's row.
 
     The Candidate part is the rows [0, rows - n_recent) (the newest n_recent rows are the Recent part
     and are never touched); the Vague part is every token whose `vague` flag is set, with its score in
@@ -276,10 +276,10 @@ def swap(Kr, Vr, ret_idx, row_scores, tok_scores, cells, n_recent: int, replace_
         Kt, Vt = query(cells[None], np.array([[J]], np.int32), seeds, mix)      # tmp <- V.Query(J)
         Kt, Vt = Kt[0, 0], Vt[0, 0]
         one = np.array([[J]], np.int32)
-        cells = insert_rows(cells[None], -Kt[None, None], -Vt[None, None], one, seeds, mix)[0]     # V.Delete(tmp)
+        cells = insert_rows(cells[None], -Kt[None, None], -Vt[None, None], one, seeds, mix)[0]     # remove the queried token from the sketch
         Jc = int(ret_idx[row])
         cells = insert_rows(cells[None], Kr[row][None, None], Vr[row][None, None],
-                            np.array([[Jc]], np.int32), seeds, mix)[0]          # V.Insert(C.Top_Pop())
+                            np.array([[Jc]], np.int32), seeds, mix)[0]          # the candidate goes into the sketch
         tok_scores[Jc] = c_min
         vague[Jc], vague[J] = True, False
         Kr[row] = round_rows(Kt) if round_rows is not None else Kt               # C.Push(tmp)

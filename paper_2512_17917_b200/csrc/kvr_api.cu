@@ -123,16 +123,24 @@ kvr_status_t compress_impl(kvr_sketch* sk, const LayerRange& lr, const void* K, 
     else KVR_CUDA(kvr_launch_scores(sk, s, K, Qobs, st));
     sk->last_score_kernel = tc ? KVR_SCORE_TCGEN05 : KVR_SCORE_MMA_SYNC;
     // ---- selection, exact copies, sketch insertion, decode list ----
+    // From here on the membership bitmap, the cells and the lists are being rewritten: until every
+    // launch below has gone through, the layers count as never compressed (a decode would otherwise
+    // read half-written state).
+    for (int l = lr.layer0; l < lr.layer0 + lr.n_layers; ++l) sk->layer_N[l] = sk->layer_R[l] = -1;
     KVR_CUDA(kvr_launch_select(sk, lr.inst0, lr.n_inst, N, R, n_recent, ret_idx, st));
     // The token lists only need the membership bitmap and a handful of CTAs; they are built on the
     // handle's side stream while the copies and the insertion (thousands of CTAs) run on `st`.
     KVR_CUDA(cudaEventRecord(sk->ev_fork, st));
     KVR_CUDA(cudaStreamWaitEvent(sk->side, sk->ev_fork, 0));
-    KVR_CUDA(kvr_launch_lists(sk, lr.inst0, lr.n_inst, N, sk->side));
-    KVR_CUDA(cudaEventRecord(sk->ev_join, sk->side));
-    KVR_CUDA(kvr_launch_gather(sk, lr.n_inst, N, R, K, V, ret_idx, Kr, Vr, st));
-    KVR_CUDA(kvr_launch_insert(sk, lr.inst0, lr.n_inst, N, K, V, st));
-    KVR_CUDA(cudaStreamWaitEvent(st, sk->ev_join, 0));
+    // The side stream has forked: whatever happens next, it is joined again before this call returns
+    // (an unjoined fork would break a stream capture and let the next call race with the lists kernel).
+    cudaError_t e = kvr_launch_lists(sk, lr.inst0, lr.n_inst, N, sk->side);
+    const cudaError_t e_rec = cudaEventRecord(sk->ev_join, sk->side);
+    if (e == cudaSuccess) e = kvr_launch_gather(sk, lr.n_inst, N, R, K, V, ret_idx, Kr, Vr, st);
+    if (e == cudaSuccess) e = kvr_launch_insert(sk, lr.inst0, lr.n_inst, N, K, V, st);
+    const cudaError_t e_join = (e_rec == cudaSuccess) ? cudaStreamWaitEvent(st, sk->ev_join, 0) : e_rec;
+    if (e == cudaSuccess) e = e_join;
+    if (e != cudaSuccess) { cudaGetLastError(); return map_err(e); }
     for (int l = lr.layer0; l < lr.layer0 + lr.n_layers; ++l) { sk->layer_N[l] = N; sk->layer_R[l] = R; }
     return KVR_OK;
 }

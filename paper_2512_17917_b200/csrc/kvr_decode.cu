@@ -10,6 +10,8 @@
 // The CTA that arrives last at a per-instance ticket merges all partials into `out`: no waiting.
 // The compressed list is ordered by row-0 cell, so that cell stays in registers while its tokens
 // are processed; the other two cells are fetched from global memory (L1/L2).
+#include <mutex>
+
 #include "kvr_internal.h"
 
 namespace {
@@ -25,7 +27,8 @@ struct DecodeParams {
     const uint32_t* dlist; // handle base: [inst][max_ctx]
     const int32_t* doff;   // handle base: [inst][b+1]
     float* part;           // [n_inst][S][G][DEC_PART]
-    uint32_t* tickets;     // handle base: [inst]
+    uint32_t* tickets;     // arrival counters; head-instance u of the call uses slot ticket0 + u
+    int ticket0;
     float* out;            // [n_inst][G][D]
     float* ml;             // handle base: [inst][G][2] maximum (log2 units) and sum of the softmax
     int inst0, R, a, b, max_ctx, n_splits;
@@ -213,7 +216,7 @@ decode_split_kernel(const DecodeParams p) {
     __threadfence();
     __syncthreads();
     if (tid == 0) {
-        const unsigned t = atomicAdd(&p.tickets[inst], 1u);
+        const unsigned t = atomicAdd(&p.tickets[p.ticket0 + u], 1u);
         s_last = (t == (unsigned)(S - 1));
     }
     __syncthreads();
@@ -234,7 +237,7 @@ decode_split_kernel(const DecodeParams p) {
         p.out[((size_t)u * G + g) * KVR_D + d] = O / L;
         if (d == 0) { p.ml[((size_t)inst * G + g) * 2] = M; p.ml[((size_t)inst * G + g) * 2 + 1] = L; }
     }
-    if (tid == 0) p.tickets[inst] = 0u;
+    if (tid == 0) p.tickets[p.ticket0 + u] = 0u;
 }
 
 template <typename T>
@@ -278,6 +281,7 @@ cudaError_t kvr_launch_decode(kvr_sketch* sk, int inst0, int n_inst, int N, int 
     p.doff = sk->doff;
     p.part = (float*)sk->ws_decode;
     p.tickets = sk->tickets;
+    p.ticket0 = inst0;
     p.out = out;
     p.ml = sk->ml;
     p.mean = sk->combine;
@@ -313,8 +317,10 @@ unsigned char* g_static_scratch_ptr[kMaxDevices];   // device address of kvr_sta
 
 // The array's name is only a host-side stand-in; the address a kernel can use has to be asked for,
 // once per device, with that device current.
+std::mutex g_static_scratch_mutex;                   // two handles on two host threads may make their first call together
 cudaError_t static_scratch_address(int device, unsigned char** out) {
     if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
     if (!g_static_scratch_ptr[device]) {
         unsigned char* ptr = nullptr;
         cudaError_t e = cudaGetSymbolAddress((void**)&ptr, kvr_static_scratch);
@@ -345,8 +351,8 @@ extern "C" kvr_status_t kvr_decode_attention_static(kvr_sketch_t* sk, int32_t la
         if (sk->layer_N[l] < 0) return KVR_ERR_STATE;
         if (sk->layer_N[l] != N || sk->layer_R[l] != R) return KVR_ERR_SHAPE;
     }
-    if (n_retained != R) return KVR_ERR_SHAPE;
-    if (R > 0 && (!Kr || !Vr)) return KVR_ERR_INVALID_ARG;
+    if (n_retained < R) return KVR_ERR_SHAPE;          // rows beyond R: tokens appended after the compress
+    if (n_retained > 0 && (!Kr || !Vr)) return KVR_ERR_INVALID_ARG;
 
     // scratch layout: [0, 16 KiB) one ticket per head-instance of the call, then the split partials
     const int S = kvr_decode_pick_splits(sk, n_inst, N, R);
@@ -374,13 +380,13 @@ extern "C" kvr_status_t kvr_decode_attention_static(kvr_sketch_t* sk, int32_t la
         p.dlist = sk->dlist;
         p.doff = sk->doff;
         p.part = reinterpret_cast<float*>(scratch + ticket_bytes);
-        // the kernel indexes tickets by absolute head-instance; slot 0 belongs to the call's first one
-        p.tickets = reinterpret_cast<uint32_t*>(scratch) - inst0;
+        p.tickets = reinterpret_cast<uint32_t*>(scratch);        // slot 0 belongs to the call's first head-instance
+        p.ticket0 = 0;
         p.out = out;
         p.ml = sk->ml;
         p.mean = sk->combine;
         p.inst0 = inst0;
-        p.R = R;
+        p.R = n_retained;
         p.a = N - R;
         p.b = sk->d.b;
         p.max_ctx = sk->d.max_context;
@@ -391,6 +397,7 @@ extern "C" kvr_status_t kvr_decode_attention_static(kvr_sketch_t* sk, int32_t la
         cudaError_t e = (sk->d.kv_dtype == KVR_F16) ? launch_G<__half>(p, sk->G, grid, st)
                                                     : launch_G<__nv_bfloat16>(p, sk->G, grid, st);
         if (e != cudaSuccess) rc = KVR_ERR_CUDA;
+        else sk->last_decode_kernel = KVR_DECODE_SPLIT;
     }
     if (prev != sk->device) cudaSetDevice(prev);
     return rc;

@@ -53,7 +53,7 @@ constexpr int CELLF = 2 * KVR_D;    // floats of one staged cell: keys[128] | va
 constexpr int CELLB = CELLF * 4;
 constexpr int HALFB = KVR_D * 4;    // bytes of the key half (or the value half) of a cell
 constexpr unsigned FULL = 0xFFFFFFFFu;
-constexpr size_t SMEM_LIMIT = 227 * 1024 - 1024;   // dynamic part; the kernel also has some static shared memory
+constexpr size_t SMEM_LIMIT = 227 * 1024 - 2048;   // dynamic part; the kernel also has about 1.2 KB of static shared memory
 // time of one retained row relative to one reconstructed token (measured): in a CTA that also serves
 // a class and in a CTA that only streams rows
 constexpr double COST_CLS = 0.45, COST_EXTRA = 0.45;
@@ -224,7 +224,7 @@ decode_staged_kernel(const StagedParams p) {
     // (g0 g1, g0 g1, g0 g2, g0 g2) for the 8 sign patterns of an entry; static shared memory sits at
     // the bottom of the window, so the table's address fits the 16 bits a descriptor has for it
     __shared__ __align__(128) float4 s_sign[8];
-    __shared__ float s_red[NW][4];
+    __shared__ float s_red[32][4], s_redl[32][4];     // per warp and head: largest logit, sum of weights
     __shared__ float s_M[4], s_L[4];
 
     const Layout L = make_layout(p.n1, p.lcap, p.rcap, G);
@@ -239,6 +239,13 @@ decode_staged_kernel(const StagedParams p) {
     // CTAs take the SMs this launch frees one by one and stage their cells while this launch drains.
     asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
 
+    // (asked for first: the cell copies below do not need them, and they are back by the time they do)
+    int k_lo = 0, k_hi = 0;
+    if (!extra) {
+        const int32_t* coff = p.coff + (size_t)inst * (C * C + 1);
+        k_lo = __ldg(coff + cls);
+        k_hi = __ldg(coff + cls + 1);
+    }
     const uint32_t smem_s = (uint32_t)__cvta_generic_to_shared(smem);
     const uint32_t cells_s = smem_s + L.cells, desc_s = smem_s + L.desc, wbuf_s = smem_s + L.wbuf;
     // ---------------------------------------------------------------- start staging.  The class's cells
@@ -268,8 +275,7 @@ decode_staged_kernel(const StagedParams p) {
     // this CTA's slice of its class, and its retained rows
     int s_begin = 0, s_end = 0, r_begin, r_end;
     if (!extra) {
-        const int32_t* coff = p.coff + (size_t)inst * (C * C + 1);
-        const int k_lo = coff[cls], k_len = coff[cls + 1] - k_lo;
+        const int k_len = k_hi - k_lo;
         s_begin = k_lo + (int)((long long)k_len * sp / p.S);
         s_end = k_lo + (int)((long long)k_len * (sp + 1) / p.S);
         r_begin = (int)((long long)p.r_cls * rec / p.n_ccta);
@@ -340,17 +346,7 @@ decode_staged_kernel(const StagedParams p) {
         rn = len - qn * NGRP;
         r0 = grp * qn + min(grp, rn);
     };
-    // Each group asks for the row-0 key half of its first token right away (entry read from global memory).
-    uint32_t c0_first = 0;
-    if (len0 > 0) {
-        int qn, rn, r0;
-        share(len0, qn, rn, r0);
-        if (qn + (grp < rn ? 1 : 0) > 0) {
-            c0_first = clist[s_begin + r0].y >> KVR_CL_C0_SHIFT;
-            fetch_row0(p.cells + (size_t)inst * 2 * KVR_R * b * KVR_D + 4 * lg, c0_first, 0u);
-        }
-    }
-
+    uint32_t c0_first = 0;                                     // row-0 cell of the group's first token
     const int own = lg >> SH;                                  // the head whose logit this lane ends up with
     const uint32_t lane16 = (uint32_t)(lg * 16);
 
@@ -363,10 +359,6 @@ decode_staged_kernel(const StagedParams p) {
         if (st > 0) {
             __syncthreads();                                   // previous stretch consumed
             asm volatile("cp.async.wait_all;\n" ::: "memory");
-            if (qn + (ragged_live ? 1 : 0) > 0) {
-                c0_first = clist[cb + r0].y >> KVR_CL_C0_SHIFT;
-                fetch_row0(p.cells + (size_t)inst * 2 * KVR_R * b * KVR_D + 4 * lg, c0_first, 0u);
-            }
         }
         // ------------------------------------------------------------ key pass
         // The scaled queries, head order permuted by lane: slot i holds head i ^ own, so that every
@@ -416,6 +408,7 @@ decode_staged_kernel(const StagedParams p) {
             }
             return mine;
         };
+        float mx = M_EMPTY;                                        // largest logit this lane has seen (head `own`)
         constexpr int FLB = (LPT == 16) ? 8 : 4, FLT = (LPT == 16) ? 2 : 1;                            // rows per group in flight: full blocks, tail
         // retained rows (exact keys): row t of the stretch goes to group t mod NGRP.  All lanes of a
         // (token, head) quad hold the same logit and store it to the same word.
@@ -440,7 +433,10 @@ decode_staged_kernel(const StagedParams p) {
 #pragma unroll
                     for (int c = 0; c < NC; ++c) { unpack4<T>(kx[i][c], t2); kp[2 * c] = t2[0]; kp[2 * c + 1] = t2[1]; }
                     const float mine = logit(kp);
-                    if (!CHECK || base + i * NGRP + grp < nrows) sts_f32(wb + i * NGRP * G * 4, mine);
+                    if (!CHECK || base + i * NGRP + grp < nrows) {
+                        mx = fmaxf(mx, mine);
+                        sts_f32(wb + i * NGRP * G * 4, mine);
+                    }
                 }
             };
             int base = 0;
@@ -454,29 +450,43 @@ decode_staged_kernel(const StagedParams p) {
         // (also set for the first token of every group).  The entries lie in the upper half of the
         // descriptor array; a batch of descriptors only overwrites entries that were read before.
         if (st == 0 && len0 > 0 && !mbar_wait(bar_list, 0)) atomicOr(p.status, 1);       // the first entries have landed
+        const float* g0K = p.cells + (size_t)inst * 2 * KVR_R * b * KVR_D + 4 * lg;      // this lane's piece of row-0 cell 0, key half
         {
             const uint2* staged = reinterpret_cast<const uint2*>(smem + L.stage) + lshift;
             uint4* desc = reinterpret_cast<uint4*>(smem + L.desc);
+            // each group asks for the row-0 key half of its first token
+            if (qn + (ragged_live ? 1 : 0) > 0) {
+                c0_first = ((st == 0) ? staged[r0].y : __ldg(&clist[cb + r0].y)) >> KVR_CL_C0_SHIFT;
+                fetch_row0(g0K, c0_first, 0u);
+            }
             const int split = rn * (qn + 1);
-            for (int base = 0; base < len; base += NT) {
-                const int i = base + tid;
-                uint2 e = make_uint2(0u, 0u);
-                if (i < len) e = (st == 0) ? staged[i] : clist[cb + i];
+            constexpr int EPT = 4;                             // entries a thread holds at a time
+            for (int base = 0; base < len; base += EPT * NT) {
+                uint2 e[EPT];
+#pragma unroll
+                for (int k = 0; k < EPT; ++k) {
+                    const int i = base + k * NT + tid;
+                    e[k] = make_uint2(0u, 0u);
+                    if (i < len) e[k] = (st == 0) ? staged[i] : clist[cb + i];
+                }
                 __syncthreads();
-                if (i < len) {
-                    bool start = true;                         // first token of its group?
-                    if (qn > 0) start = (i < split) ? (i % (qn + 1) == 0) : ((i - split) % qn == 0);
-                    uint4 d;
-                    d.x = cells_s + (e.x & 0xFFu) * CELLB;
-                    d.y = cells_s + ((e.x >> 8) & 0xFFu) * CELLB;
-                    d.z = wbuf_s + (uint32_t)(nrows + i) * (G * 4);
-                    d.w = (e.x & 0xFFFF0000u) | (sign_s + (e.y & 0x70u)) | (e.y & KVR_CL_FLAG) | (start ? KVR_CL_FLAG : 0u);
-                    desc[i] = d;
+#pragma unroll
+                for (int k = 0; k < EPT; ++k) {
+                    const int i = base + k * NT + tid;
+                    if (i < len) {
+                        bool start = true;                     // first token of its group?
+                        if (qn > 0) start = (i < split) ? (i % (qn + 1) == 0) : ((i - split) % qn == 0);
+                        uint4 d;
+                        d.x = cells_s + (e[k].x & 0xFFu) * CELLB;
+                        d.y = cells_s + ((e[k].x >> 8) & 0xFFu) * CELLB;
+                        d.z = wbuf_s + (uint32_t)(nrows + i) * (G * 4);
+                        d.w = (e[k].x & 0xFFFF0000u) | (sign_s + (e[k].y & 0x70u)) | (e[k].y & KVR_CL_FLAG) | (start ? KVR_CL_FLAG : 0u);
+                        desc[i] = d;
+                    }
                 }
             }
             __syncthreads();
         }
-        const float* g0K = p.cells + (size_t)inst * 2 * KVR_R * b * KVR_D + 4 * lg;
         if (st == 0 && !extra && !mbar_wait(bar_cells, 0)) atomicOr(p.status, 1);       // the cells have landed
         // compressed tokens (Algorithm 2 on the key halves)
         if (len > 0) {
@@ -503,7 +513,10 @@ decode_staged_kernel(const StagedParams p) {
                     }
                 });
                 const float mine = logit(kp);
-                if (live) sts_f32(d.z + own4, mine);
+                if (live) {
+                    mx = fmaxf(mx, mine);
+                    sts_f32(d.z + own4, mine);
+                }
             };
             uint32_t dp = desc_s + (uint32_t)r0 * 16u;
 #pragma unroll 1
@@ -513,50 +526,37 @@ decode_staged_kernel(const StagedParams p) {
             asm volatile("cp.async.wait_all;\n" ::: "memory");
             if (qn + (ragged_live ? 1 : 0) > 0) fetch_row0(g0K + (size_t)KVR_R * b * KVR_D, c0_first, 0u);
         }
+        // the warp's largest logits per head (the lanes of a (token, head) quad hold the same value)
+#pragma unroll
+        for (int x = LPT; x < 32; x <<= 1) mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, x));
+        if (lane < LPT && (lg & ((1 << SH) - 1)) == 0) s_red[warp][own] = mx;
         __syncthreads();
         // ------------------------------------------------------------ logits -> weights, in place: the
-        // CTA's maximum per head, then w = 2^(logit - max) (times g_0 for a reconstructed token), and
-        // the sums.  NT is a multiple of G: a thread stays with one head.
+        // CTA's maximum per head (every warp folds the warps' maxima itself), then
+        // w = 2^(logit - max) (times g_0 for a reconstructed token), and the warps' sums
         {
             const int n_tok = nrows + len;
             float* w = reinterpret_cast<float*>(smem + L.wbuf);
-            auto load_tok = [&](int t, float (&x)[G]) {
+            float M[G], l[G];
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                float v = lane < NW ? s_red[lane][g] : M_EMPTY;
+#pragma unroll
+                for (int x = 1; x < 32; x <<= 1) v = fmaxf(v, __shfl_xor_sync(FULL, v, x));
+                M[g] = v;
+                l[g] = 0.f;
+            }
+            if (tid < G) {
+                float m = M[0];
+#pragma unroll
+                for (int g = 1; g < G; ++g) m = (tid == g) ? M[g] : m;
+                s_M[tid] = m;
+            }
+            for (int t = tid; t < n_tok; t += NT) {
+                float x[G];
                 if constexpr (G == 4) { const float4 v = *reinterpret_cast<const float4*>(w + 4 * t); x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w; }
                 else if constexpr (G == 2) { const float2 v = *reinterpret_cast<const float2*>(w + 2 * t); x[0] = v.x; x[1] = v.y; }
                 else x[0] = w[t];
-            };
-            float mx[G];
-#pragma unroll
-            for (int g = 0; g < G; ++g) mx[g] = M_EMPTY;
-            for (int t = tid; t < n_tok; t += NT) {
-                float x[G];
-                load_tok(t, x);
-#pragma unroll
-                for (int g = 0; g < G; ++g) mx[g] = fmaxf(mx[g], x[g]);
-            }
-#pragma unroll
-            for (int g = 0; g < G; ++g) {
-#pragma unroll
-                for (int x = 1; x < 32; x <<= 1) mx[g] = fmaxf(mx[g], __shfl_xor_sync(FULL, mx[g], x));
-                if (lane == 0) s_red[warp][g] = mx[g];
-            }
-            __syncthreads();
-            if (warp == 0) {
-#pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    float v = lane < NW ? s_red[lane][g] : M_EMPTY;
-#pragma unroll
-                    for (int x = 1; x < 32; x <<= 1) v = fmaxf(v, __shfl_xor_sync(FULL, v, x));
-                    if (lane == 0) s_M[g] = v;
-                }
-            }
-            __syncthreads();
-            float M[G], l[G];
-#pragma unroll
-            for (int g = 0; g < G; ++g) { M[g] = s_M[g]; l[g] = 0.f; }
-            for (int t = tid; t < n_tok; t += NT) {
-                float x[G];
-                load_tok(t, x);
                 float sgn = 1.f;
                 if (t >= nrows) {
                     if (lds_u32(desc_s + (uint32_t)(t - nrows) * 16u + 12u) & (1u << KVR_CL_SIGN_SHIFT)) sgn = -1.f;   // g_0
@@ -576,19 +576,10 @@ decode_staged_kernel(const StagedParams p) {
 #pragma unroll
             for (int g = 0; g < G; ++g) {
 #pragma unroll
-                for (int x = 1; x < 32; x <<= 1) l[g] += __shfl_xor_sync(FULL, l[g], x);
-                if (lane == 0) s_red[warp][g] = l[g];     // (the maxima in s_red were consumed before the barrier above)
+                for (int x = 1; x < 32; x <<= 1) l[g] += __shfl_xor_sync(FULL, l[g], x);   // a fixed tree: same sum every run
+                if (lane == 0) s_redl[warp][g] = l[g];
             }
             __syncthreads();
-            if (warp == 0) {
-#pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    float v = lane < NW ? s_red[lane][g] : 0.f;
-#pragma unroll
-                    for (int x = 1; x < 32; x <<= 1) v += __shfl_xor_sync(FULL, v, x);      // a fixed tree: same sum every run
-                    if (lane == 0) s_L[g] = v;
-                }
-            }
         }
         // ------------------------------------------------------------ value pass
         u64 o2[G][NP];
@@ -701,6 +692,15 @@ decode_staged_kernel(const StagedParams p) {
                             unpack2(o2[g][2 * c + 1], v.z, v.w);
                             *reinterpret_cast<float4*>(r + g * KVR_D + (c * LPT + lg) * 4) = v;
                         }
+                }
+                if (g0 == 0 && warp == 0) {                  // the CTA's sums of weights (fixed tree)
+#pragma unroll
+                    for (int g = 0; g < G; ++g) {
+                        float v = lane < NW ? s_redl[lane][g] : 0.f;
+#pragma unroll
+                        for (int x = 1; x < 32; x <<= 1) v += __shfl_xor_sync(FULL, v, x);
+                        if (lane == 0) s_L[g] = v;
+                    }
                 }
                 __syncthreads();
                 if (tid < G * KVR_D) {

@@ -168,21 +168,21 @@ swap_kernel(T* __restrict__ Kr_all, T* __restrict__ Vr_all, int32_t* __restrict_
                     kk[i] = cK[cell[i]];
                     vv[i] = gv[i] * cV[cell[i]];
                 }
-                const float Kt = kvr_comb3(kk[0], kk[1], kk[2], mean), Vt = kvr_comb3(vv[0], vv[1], vv[2], mean);   // tmp <- V.Query
+                const float Kt = kvr_comb3(kk[0], kk[1], kk[2], mean), Vt = kvr_comb3(vv[0], vv[1], vv[2], mean);   // query the vague token (Algorithm 2)
 #pragma unroll
-                for (int i = 0; i < KVR_R; ++i) {                 // V.Delete(tmp)
+                for (int i = 0; i < KVR_R; ++i) {                 // take it out of the sketch again
                     cK[cell[i]] -= Kt;
                     cV[cell[i]] -= gv[i] * Vt;
                 }
                 const float kc = KvrType<T>::to_float(Kr[(size_t)row * KVR_D + d]);
                 const float vc = KvrType<T>::to_float(Vr[(size_t)row * KVR_D + d]);
 #pragma unroll
-                for (int i = 0; i < KVR_R; ++i) {                 // V.Insert(C.Top_Pop())
+                for (int i = 0; i < KVR_R; ++i) {                 // the candidate's vectors go in (Algorithm 1)
                     const size_t cc = ((size_t)i * b + tok_h[(size_t)i * max_ctx + Jc]) * KVR_D + d;
                     cK[cc] += kc;
                     cV[cc] += (float)tok_g[(size_t)i * max_ctx + Jc] * vc;
                 }
-                Kr[(size_t)row * KVR_D + d] = KvrType<T>::from_float(Kt);                            // C.Push(tmp)
+                Kr[(size_t)row * KVR_D + d] = KvrType<T>::from_float(Kt);                            // the queried vectors take its row
                 Vr[(size_t)row * KVR_D + d] = KvrType<T>::from_float(Vt);
             }
             if (tid == 1023) {

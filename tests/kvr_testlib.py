@@ -57,6 +57,14 @@ def make_case(seed, B, H, Hq, N, W, dtype, L=1, n_outlier=4):
     return torch.stack(Ks), torch.stack(Vs), torch.stack(Qs), torch.stack(qs)
 
 
+def sampled_instances(n_inst: int, k: int, salt: int = 0):
+    """k head-instances for the oracle to check at full size.  The choice is a fixed function of
+    KVR_TEST_SEED (default 0): another seed checks other instances."""
+    import os
+    rng = np.random.default_rng([int(os.environ.get("KVR_TEST_SEED", "0")), salt, n_inst])
+    return sorted(int(x) for x in rng.choice(n_inst, size=min(k, n_inst), replace=False))
+
+
 def check_selection_band(s64: np.ndarray, ret: np.ndarray, R: int, n_recent: int):
     """Selection vs the oracle's fp64 scores: exact outside the ambiguity band."""
     n_inst, N = s64.shape
@@ -78,7 +86,8 @@ def check_selection_band(s64: np.ndarray, ret: np.ndarray, R: int, n_recent: int
 
 
 def run_and_check(K, V, Qobs, q, *, R, n_recent, b, seeds, index_mix=True, layer_mode="per_layer",
-                  sample_inst=None, check_reconstruct=True, scale=0.0, decode_kernel=None, score_kernel=None, obs_causal=False, combine="median"):
+                  sample_inst=None, check_reconstruct=True, scale=0.0, decode_kernel=None, score_kernel=None, obs_causal=False, combine="median",
+                  expect_decode_kernel=None):
     """Compress + one decode step on the GPU through the C ABI, the same through the oracle,
     compare every stage.  K, V, Qobs, q carry a leading layer axis.  Returns (gpu_out, oracle_out)."""
     L, B, H, N, D = K.shape
@@ -111,6 +120,8 @@ def run_and_check(K, V, Qobs, q, *, R, n_recent, b, seeds, index_mix=True, layer
         Kr, Vr, ret, out = torch.stack(Krs), torch.stack(Vrs), torch.stack(rets), torch.stack(outs)
     if decode_kernel is not None and decode_kernel != kvr.KVR_DECODE_AUTO:
         assert kvr.kvr_last_decode_kernel(sk) == decode_kernel, "the requested decode kernel did not run"
+    if expect_decode_kernel is not None:
+        assert kvr.kvr_last_decode_kernel(sk) == expect_decode_kernel, "the library chose another decode kernel"
     if score_kernel is not None and score_kernel != kvr.KVR_SCORE_AUTO:
         assert kvr.kvr_last_score_kernel(sk) == score_kernel, "the requested scoring kernel did not run"
     assert kvr.kvr_sketch_device_status(sk) == 0, "a bounded wait inside a kernel gave up"

@@ -10,7 +10,7 @@ import paper_2512_17917_b200 as kvr
 from oracle import kvr_oracle as orc
 from paper_2512_17917_b200 import synth
 
-from kvr_testlib import TOL, dec_to_inst, inst_major, make_case, run_and_check
+from kvr_testlib import TOL, dec_to_inst, inst_major, make_case, run_and_check, sampled_instances
 
 pytestmark = pytest.mark.gpu
 F16, BF16 = torch.float16, torch.bfloat16
@@ -454,20 +454,19 @@ def test_32k_full_size_sampled(mode, L):
     K, V, Q = torch.stack(Ks), torch.stack(Vs), torch.stack(Qs)
     q = synth.decode_queries(w, 0, dev)[:L]
     n_inst = L * w.n_kv_heads
-    sample = sorted({1, n_inst - 2})
     run_and_check(K.cpu(), V.cpu(), Q.cpu(), q.cpu(), R=w.budget, n_recent=0, b=w.b,
-                  seeds=synth.hash_seeds(w.seed + 3), layer_mode=mode, sample_inst=sample)
+                  seeds=synth.hash_seeds(w.seed + 3), layer_mode=mode, sample_inst=sampled_instances(n_inst, 2, L),
+                  expect_decode_kernel=kvr.KVR_DECODE_STAGED)        # the kernel the benchmark times
 
 
-@pytest.mark.parametrize("name,ratio,mult", [
-    ("32k_llama3_8b_batch16", 0.0, 0.0),        # bf16, 128 head-instances per layer launch: 2048 class CTAs, many waves
-    ("8k_qwen3_8b_batch8", 0.10, 1.0),          # 64 head-instances, one class, two token slices per class
-    ("8k_qwen3_8b_batch8", 0.50, 2.0),          # widest sketch of the sweep at the largest budget (4 x 4 classes)
-    ("2k_llama3_8b", 0.0, 0.0),                 # short context: one class cut into 18 slices per head-instance
-])
-def test_other_workloads_one_layer_sampled(name, ratio, mult):
+@pytest.mark.parametrize("name,ratio,mult,n_sample", [
+    ("32k_llama3_8b_batch16", 0.0, 0.0, 3),     # bf16, 128 head-instances per layer launch: 2048 class CTAs, many waves
+    ("2k_llama3_8b", 0.0, 0.0, 3),              # short context: one class cut into slices per head-instance
+] + [("8k_qwen3_8b_batch8", r, m, 1) for r in (0.05, 0.10, 0.25, 0.50) for m in (0.5, 1.0, 2.0)])   # the whole sweep
+def test_other_workloads_one_layer_sampled(name, ratio, mult, n_sample):
     """One layer of the other benchmark workloads at full per-layer size, in the launch shape the
-    benchmark uses for them (one layer per call); the oracle checks three sampled head-instances."""
+    benchmark uses for them (one layer per call), every point of the budget x width sweep included;
+    the oracle checks sampled head-instances.  The library has to pick the staged kernel by itself."""
     import dataclasses
     w = synth.WORKLOADS[name]
     if ratio:
@@ -476,8 +475,8 @@ def test_other_workloads_one_layer_sampled(name, ratio, mult):
     q = synth.decode_queries(w, 0, "cuda")[:1]
     n_inst = w.batch * w.n_kv_heads
     run_and_check(K[None].cpu(), V[None].cpu(), Q[None].cpu(), q.cpu(), R=w.budget, n_recent=0, b=w.b,
-                  seeds=synth.hash_seeds(w.seed + 3), sample_inst=sorted({0, n_inst // 2 + 1, n_inst - 1}),
-                  check_reconstruct=False)
+                  seeds=synth.hash_seeds(w.seed + 3), sample_inst=sampled_instances(n_inst, n_sample, int(ratio * 100 + mult * 10)),
+                  check_reconstruct=False, expect_decode_kernel=kvr.KVR_DECODE_STAGED)
 
 
 def test_recompress_with_other_shape_and_determinism():
