@@ -289,6 +289,66 @@ def swap(Kr, Vr, ret_idx, row_scores, tok_scores, cells, n_recent: int, replace_
     return Kr, Vr, ret_idx, row_scores, tok_scores, cells, n_swaps
 
 
+def append_sizes(n_rows: int, n_recent: int, n_new: int, r_budget: int, c_budget: int, slack: int):
+    """Sizes after Algorithm 3 has taken n_new tokens (counting only; no data is looked at): returns
+    (rows_after, recent_after).  The Recent part gives up its oldest tokens only once it exceeds its
+    budget by more than Slack, and then all of its excess at once; the Candidate part never keeps more
+    than its budget."""
+    recent = n_recent + n_new
+    cand = n_rows - n_recent
+    if recent > r_budget + slack:
+        cand += recent - r_budget
+        recent = r_budget
+    return min(cand, c_budget) + recent, recent
+
+
+def compress_stream(Kr, Vr, ret_idx, row_scores, n_recent: int, tok_scores, cells, K_new, V_new, idx_new,
+                    r_budget: int, c_budget: int, slack: int, replace_rate: float, max_swaps: int,
+                    seeds, mix: bool = True, round_rows=None):
+    """Algorithm 3 (insert newly generated tokens and compress) for ONE head-instance, in the
+    algorithm's order:
+      1. the new tokens are pushed to the Recent part (a queue, oldest first; they arrive with score 0);
+      2. if the Recent part now exceeds its budget by more than Slack, its oldest tokens, all that
+         exceed the budget, move to the Candidate part in one go;
+      3. while the Candidate part is over its budget, its lowest-scored token is taken out and inserted
+         into the sketch (Algorithm 1); among equal scores the newest goes first, so that the older
+         token stays (the same rule as `demote`); the token's score moves to the per-token array;
+      4. the swap loop (`swap`).
+    The storage is the exact rows in order: Candidate rows first, then the n_recent Recent rows.
+    Arguments as in `swap`, plus K_new, V_new [n_new, D] and their token indices idx_new [n_new].
+    Everything is updated on copies; returns
+    (Kr, Vr, ret_idx, row_scores, n_recent, tok_scores, cells, n_swaps)."""
+    Kr, Vr = np.array(Kr, np.float64), np.array(Vr, np.float64)
+    ret_idx, row_scores = np.array(ret_idx, np.int32), np.array(row_scores, np.float32)
+    tok_scores = np.array(tok_scores, np.float32)
+    cells = np.array(cells, np.float64, copy=True, order="C")
+    K_new, V_new = np.array(K_new, np.float64), np.array(V_new, np.float64)
+    rows = [dict(k=Kr[i], v=Vr[i], idx=int(ret_idx[i]), score=np.float32(row_scores[i])) for i in range(len(ret_idx))]
+    cut = len(rows) - n_recent
+    C, R = rows[:cut], rows[cut:]
+    for j in range(len(idx_new)):                                                # 1. R.Push(T)
+        R.append(dict(k=K_new[j], v=V_new[j], idx=int(idx_new[j]), score=np.float32(0.0)))
+    if len(R) > r_budget + slack:                                                # 2. R over budget + Slack
+        k = len(R) - r_budget
+        C.extend(R[:k])
+        R = R[k:]
+    while len(C) > c_budget:                                                     # 3. pop the minimum into the sketch
+        lo = min(range(len(C)), key=lambda i: (C[i]["score"], -i))
+        t = C.pop(lo)
+        one = np.array([[t["idx"]]], np.int32)
+        cells = insert_rows(cells[None], t["k"][None, None], t["v"][None, None], one, seeds, mix)[0]
+        tok_scores[t["idx"]] = t["score"]
+    rows = C + R
+    D = Kr.shape[1] if Kr.ndim == 2 else K_new.shape[1]
+    Kr2 = np.array([t["k"] for t in rows], np.float64).reshape(len(rows), D)
+    Vr2 = np.array([t["v"] for t in rows], np.float64).reshape(len(rows), D)
+    ret2 = np.array([t["idx"] for t in rows], np.int32)
+    sc2 = np.array([t["score"] for t in rows], np.float32)
+    Kr2, Vr2, ret2, sc2, tok_scores, cells, n = swap(Kr2, Vr2, ret2, sc2, tok_scores, cells, len(R), replace_rate,
+                                                      max_swaps, seeds, mix, round_rows)        # 4. swap loop
+    return Kr2, Vr2, ret2, sc2, len(R), tok_scores, cells, n
+
+
 def paper_split(context: int, ratio: float, r: int = 3):
     """Storage split of the paper's hyper-parameter section: Recent 0.45, Candidate 0.45, Vague 0.10 of
     the budget, r = 3 rows, the width b fixed by the Vague share once r is set; one cell counts like one

@@ -510,6 +510,106 @@ def test_swap_rate_and_limit():
     np.testing.assert_allclose(out[5], step[0], rtol=0, atol=1e-12)
 
 
+def _stream_case(seed, N=40, n_total=64, D=8, b=5, R=14, n_recent=4, injective=False):
+    Q = _rand((1, 8, D), seed)
+    K, V = _rand((1, n_total, D), seed + 1), _rand((1, n_total, D), seed + 2)
+    seeds = synth.injective_seeds() if injective else synth.hash_seeds(seed + 3)
+    bb = n_total if injective else b
+    c = orc.compress(Q, K[:, :N], V[:, :N], R=R, n_recent=n_recent, seeds=seeds, b=bb, mix=not injective)
+    return K, V, seeds, bb, c, c["scores32"][0].copy()         # per-token scores of the N tokens that exist so far
+
+
+def test_compress_stream_equals_overflow_step_then_swap_loop():
+    """Algorithm 3 taken step by step (push, bulk move out of the Recent part, pops of the minimum one
+    at a time, swap loop) against the two building blocks pinned above: the pops, for a fixed score
+    array, leave the same rows as the top-k rule of `demote` (older token kept among equals), insertion
+    is linear so the order of the pops does not matter to the cells, and the swap loop is `swap`."""
+    K, V, seeds, b, c, tok = _stream_case(700)
+    N, n_new, R, n_recent = 40, 9, 14, 4
+    rng = np.random.default_rng(701)
+    rows = (rng.random(R) ** 2).astype(np.float32)
+    rows[2] = rows[6]                                             # a tie among candidates
+    tok = np.concatenate([rng.random(N).astype(np.float32), np.zeros(n_new, np.float32)])   # vague tokens with fresh scores
+    tok[c["ret_idx"][0]] = rows
+    r_budget, c_budget, slack = 6, 8, 3                           # 4 + 9 = 13 > 6 + 3: the Recent part overflows
+    idx_new = np.arange(N, N + n_new, dtype=np.int32)
+    got = orc.compress_stream(c["Kr"][0], c["Vr"][0], c["ret_idx"][0], rows, n_recent, tok, c["cells"][0],
+                              K[0, N:N + n_new], V[0, N:N + n_new], idx_new, r_budget, c_budget, slack, 1.1, 50, seeds)
+    # the same through demote + swap
+    Kc = np.concatenate([c["Kr"], K[:, N:N + n_new]], axis=1)
+    Vc = np.concatenate([c["Vr"], V[:, N:N + n_new]], axis=1)
+    rc = np.concatenate([c["ret_idx"], idx_new[None]], axis=1)
+    sc = np.concatenate([rows, np.zeros(n_new, np.float32)])[None]
+    n_after, rec_after = orc.append_sizes(R, n_recent, n_new, r_budget, c_budget, slack)
+    assert (n_after, rec_after) == (c_budget + r_budget, r_budget)
+    keep, evict, cells2 = orc.demote(Kc, Vc, rc, sc, c["cells"], n_after, rec_after, seeds)
+    tok2 = tok.copy()
+    tok2[rc[0][evict[0]]] = sc[0][evict[0]]
+    want = orc.swap(Kc[0][keep[0]], Vc[0][keep[0]], rc[0][keep[0]], sc[0][keep[0]], tok2, cells2[0], rec_after, 1.1, 50, seeds)
+    assert got[4] == rec_after and got[7] == want[6] and got[7] > 0
+    for a_, b_ in zip(got[:4], want[:4]):
+        np.testing.assert_array_equal(a_, b_)
+    np.testing.assert_array_equal(got[5], want[4])
+    np.testing.assert_allclose(got[6], want[5], rtol=0, atol=1e-11)
+
+
+def test_compress_stream_slack_holds_the_recent_part_and_sizes_follow_the_counting_rule():
+    """Several Slack periods, one or two tokens per call: the Recent part grows until it exceeds its
+    budget by more than Slack, then drops to its budget in one go; the Candidate part never exceeds its
+    budget; `append_sizes` predicts every size from the counts alone; the retained tokens are distinct
+    and the newest tokens are always the Recent rows."""
+    K, V, seeds, b, c, tok = _stream_case(710, N=40, n_total=64)
+    Kr, Vr, ret, n_recent = c["Kr"][0], c["Vr"][0], c["ret_idx"][0], 4
+    rows = tok[ret].copy()
+    cells, ctx = c["cells"][0], 40
+    r_budget, c_budget, slack = 4, 10, 5
+    seen_drop = 0
+    rng = np.random.default_rng(711)
+    while ctx < 64:
+        n_new = min(int(rng.integers(1, 3)), 64 - ctx)
+        want_rows, want_recent = orc.append_sizes(len(ret), n_recent, n_new, r_budget, c_budget, slack)
+        rows = rows + (rng.random(len(rows)) * 0.1).astype(np.float32)           # scores keep accumulating
+        tok = np.concatenate([tok + (rng.random(len(tok)) * 0.1).astype(np.float32), np.zeros(n_new, np.float32)])
+        before_recent = n_recent
+        Kr, Vr, ret, rows, n_recent, tok, cells, _ = orc.compress_stream(
+            Kr, Vr, ret, rows, n_recent, tok, cells, K[0, ctx:ctx + n_new], V[0, ctx:ctx + n_new],
+            np.arange(ctx, ctx + n_new, dtype=np.int32), r_budget, c_budget, slack, 1.1, 10, seeds)
+        ctx += n_new
+        assert (len(ret), n_recent) == (want_rows, want_recent)
+        assert n_recent <= r_budget + slack and len(ret) - n_recent <= c_budget
+        if n_recent < before_recent + n_new:
+            assert before_recent + n_new > r_budget + slack and n_recent == r_budget
+            seen_drop += 1
+        assert len(set(ret.tolist())) == len(ret)
+        assert (ret[len(ret) - n_recent:] == np.arange(ctx - n_recent, ctx)).all()
+    assert seen_drop >= 3                                          # at least three Slack periods were run
+
+
+def test_compress_stream_under_injective_hashing_is_exact():
+    """One cell per token: whatever the history of pushes, pops and swaps, every stored row is the
+    token's own vectors and the cells equal a sketch built in one go from the final vague set."""
+    K, V, seeds, b, c, tok = _stream_case(720, injective=True)
+    Kr, Vr, ret, n_recent = c["Kr"][0], c["Vr"][0], c["ret_idx"][0], 4
+    rows, cells, ctx = tok[ret].copy(), c["cells"][0], 40
+    rng = np.random.default_rng(721)
+    swaps = 0
+    while ctx < 64:
+        n_new = min(3, 64 - ctx)
+        tok = np.concatenate([tok + (rng.random(len(tok)) * 0.5).astype(np.float32), np.zeros(n_new, np.float32)])
+        rows = rows + (rng.random(len(rows)) * 0.05).astype(np.float32)
+        Kr, Vr, ret, rows, n_recent, tok, cells, n = orc.compress_stream(
+            Kr, Vr, ret, rows, n_recent, tok, cells, K[0, ctx:ctx + n_new], V[0, ctx:ctx + n_new],
+            np.arange(ctx, ctx + n_new, dtype=np.int32), 4, 10, 2, 1.1, 10, seeds, mix=False)
+        ctx += n_new
+        swaps += n
+        np.testing.assert_allclose(Kr, K[0][ret], rtol=0, atol=1e-11)
+        np.testing.assert_allclose(Vr, V[0][ret], rtol=0, atol=1e-11)
+        vague = np.setdiff1d(np.arange(ctx), ret).astype(np.int32)
+        want = orc.insert(K[:, :ctx], V[:, :ctx], vague[None], seeds, b, mix=False)[0]
+        np.testing.assert_allclose(cells, want, rtol=0, atol=1e-11)
+    assert swaps > 0
+
+
 def test_window_scores_match_library_softmax_under_the_causal_mask():
     """In-context observation window: row (head g, query t) is token N - W + t and sees keys up to
     itself.  Against a library softmax with the mask written out; every row still sums to one, so the
