@@ -354,6 +354,69 @@ def run_gpu(args, w, rank, world, local):
     return result, (Kall, Vall, Qall, qs)
 
 
+# ------------------------------------------------------------------- streaming generation (Algorithm 3)
+def run_stream(args, w):
+    """--stream T: after the compress, T generation steps; every step and layer runs the decode over
+    the current storage, adds the step's attention mass to the scores of the stored rows and of the
+    vague tokens, and takes the new token through Algorithm 3 (kvr_append: Recent part with Slack,
+    pops into the sketch, swap loop with ReplaceRate 1.1).  One JSON line: generation tokens/s."""
+    import paper_2512_17917_b200 as kvr
+
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    L, B, H, Hq, D, N, R, T = w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, w.head_dim, w.context, w.budget, args.stream
+    dt = w.torch_dtype
+    r_budget = max(1, int(0.5 * R)) if w.n_recent else 64          # Recent budget (the storage-split preset keeps half)
+    c_budget, slack, n_recent = R - min(r_budget, R), 32, w.n_recent
+    sk = kvr.kvr_sketch_create(b=w.b, batch=B, n_layers=L, n_kv_heads=H, n_q_heads=Hq, max_context=N + T, kv_dtype=dt,
+                               hash_seeds=synth.hash_seeds(w.seed + 3), device=dev)
+    st = []
+    for layer in range(L):
+        K, V, Q = synth.layer_inputs(w, layer, dev)
+        Kr, Vr, ret = kvr.kvr_compress(sk, layer, K, V, Q, R, n_recent)
+        sc = torch.gather(kvr.kvr_get_scores(sk, layer), -1, ret.long()).contiguous()
+        st.append([Kr, Vr, ret, sc, n_recent])
+        del K, V, Q
+    gen = torch.Generator(device=dev).manual_seed(w.seed + 99)
+    new_k = (torch.randn((T, L, B, H, 1, D), generator=gen, device=dev)).to(dt)
+    new_v = (torch.randn((T, L, B, H, 1, D), generator=gen, device=dev)).to(dt)
+    qs = torch.stack([synth.decode_queries(w, s % max(1, w.decode_steps), dev) for s in range(T)])
+    out = torch.empty((B, Hq, D), dtype=torch.float32, device=dev)
+
+    def step(t):
+        for layer in range(L):
+            Kr, Vr, ret, sc, nr = st[layer]
+            kvr.kvr_decode_attention(sk, layer, qs[t, layer], Kr, Vr, ret, out=out)
+            kvr.kvr_accumulate_scores(sk, layer, qs[t, layer], Kr, sc)
+            kvr.kvr_accumulate_vague_scores(sk, layer, qs[t, layer])
+            Kr, Vr, ret, sc, nr, _ = kvr.kvr_append(sk, layer, Kr, Vr, ret, sc, nr, new_k[t, layer], new_v[t, layer],
+                                                    r_budget, c_budget, slack, 1.1, 64)
+            st[layer] = [Kr, Vr, ret, sc, nr]
+
+    warm = min(3, T // 4)
+    for t in range(warm):
+        step(t)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l0 = kvr.kvr_launch_count(sk)
+    e0.record()
+    for t in range(warm, T):
+        step(t)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / (T - warm)
+    assert kvr.kvr_sketch_device_status(sk) == 0 and torch.isfinite(out).all()
+    res = {"metric": "stream_generation_tokens_per_s", "value": round(B / (ms * 1e-3), 2), "unit": UNIT, "n_gpus": 1,
+           "steps": T - warm, "warmup": warm, "ms_per_step": round(ms, 3), "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+           "config": dict(config_of(w), launch="eager, per layer: decode + accumulate x2 + kvr_append",
+                          r_budget=r_budget, c_budget=c_budget, slack=slack, replace_rate=1.1),
+           "rows_after": int(st[0][0].shape[-2]), "context_after": N + T,
+           "gpu_launches": int(kvr.kvr_launch_count(sk) - l0)}
+    kvr.kvr_sketch_destroy(sk)
+    return res
+
+
 # ----------------------------------------------------------------------------- the CPU oracle
 def oracle_sample(w, n_sample: int, decode_steps: int, inputs=None, combine: str = "median"):
     """Time the oracle, as it stands, on n_sample head-instances of layer 0: one compress and
@@ -424,6 +487,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="kvr", choices=["kvr", "reference"])
+    ap.add_argument("--stream", type=int, default=0, help="time T generation steps with Algorithm 3 (kvr_append) instead")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling a small case)")
@@ -470,6 +534,9 @@ def main():
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback of the hot path)")
+    if args.stream > 0:
+        print(json.dumps(run_stream(args, w)), flush=True)
+        return
     if args.warmup < 3:
         args.warmup = 3
     rank, world, local = kdist.init_from_env()

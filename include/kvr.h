@@ -306,6 +306,34 @@ int32_t kvr_last_score_kernel(const kvr_sketch_t* sk);
  * handle so far completed normally; anything else means outputs since then are invalid. */
 kvr_status_t kvr_sketch_device_status(kvr_sketch_t* sk, int32_t* status, void* cuda_stream);
 
+/* Algorithm 3 ("insert newly generated token(s) T and compress") as one call.  The caller's exact
+ * storage of the layer holds n_rows rows per head-instance, the Candidate part first, the newest
+ * n_recent rows being the Recent part.  In the algorithm's order:
+ *   1. the n_new new tokens (K_new, V_new [batch, n_kv_heads, n_new, head_dim], kv_dtype) join the
+ *      Recent part; their token indices continue the context, their scores start at 0;
+ *   2. when the Recent part then holds more than r_budget + slack tokens, its oldest tokens, all that
+ *      exceed r_budget, move to the Candidate part at once;
+ *   3. while the Candidate part holds more than c_budget rows its lowest-scored row goes into the
+ *      sketch (Algorithm 1; among equal scores the older token stays), its score into the handle's
+ *      per-token array;
+ *   4. the swap loop (as kvr_swap, with replace_rate and max_swaps).
+ * How many rows remain depends on the counts only: kvr_append_sizes returns the rows (and through
+ * n_recent_after the Recent rows) the storage holds afterwards, -1 for impossible counts; the caller
+ * sizes Kr_out, Vr_out [batch, n_kv_heads, rows_after, head_dim], ret_idx_out and row_scores_out
+ * [.., rows_after] with it (they must not alias the inputs).  Nothing is waited for between the
+ * steps: every launch is enqueued on `cuda_stream`, the swap loop decides on the device.
+ * n_swapped: device [batch, n_kv_heads] int32 or NULL.  After the call the handle describes the new
+ * storage: pass rows_after to kvr_decode_attention.  Errors: INVALID_ARG, SHAPE (n_rows below the
+ * layer's retained count, context beyond max_context), STATE, ALLOC, CUDA. */
+int32_t kvr_append_sizes(int32_t n_rows, int32_t n_recent, int32_t n_new, int32_t r_budget, int32_t c_budget,
+                         int32_t slack, int32_t* n_recent_after);
+kvr_status_t kvr_append(kvr_sketch_t* sk, int32_t layer, const void* Kr, const void* Vr,
+                        const int32_t* ret_idx, const float* row_scores, int32_t n_rows, int32_t n_recent,
+                        const void* K_new, const void* V_new, int32_t n_new, int32_t r_budget,
+                        int32_t c_budget, int32_t slack, float replace_rate, int32_t max_swaps,
+                        void* Kr_out, void* Vr_out, int32_t* ret_idx_out, float* row_scores_out,
+                        int32_t* n_swapped, void* cuda_stream);
+
 /* Host-buffer forms of the two calls: inputs are copied host -> device inside the call, the
  * retained rows stay in a handle-owned device store (so Kr / Vr / ret_idx are not passed), and
  * the decode output is copied back to `out` before the call returns (it synchronises the stream).

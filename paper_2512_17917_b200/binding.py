@@ -15,6 +15,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libkvr.so")
 
 KVR_OK = 0
+KVR_ERR_SHAPE = 3
 KVR_F16, KVR_BF16 = 0, 1
 KVR_ALL_LAYERS = -1
 KVR_MAX_B = 8192
@@ -31,7 +32,7 @@ EXPORTS = (
     "kvr_sketch_set_decode_kernel", "kvr_last_decode_kernel", "kvr_sketch_device_status",
     "kvr_accumulate_scores", "kvr_demote", "kvr_sketch_set_score_kernel", "kvr_last_score_kernel",
     "kvr_accumulate_vague_scores", "kvr_swap", "kvr_sketch_set_obs_window_causal", "kvr_paper_storage_split", "kvr_layer_budgets", "kvr_sketch_set_combine",
-    "kvr_measure_pipe_peaks",
+    "kvr_measure_pipe_peaks", "kvr_append", "kvr_append_sizes",
 )
 
 
@@ -94,6 +95,9 @@ def lib() -> ctypes.CDLL:
         L.kvr_last_score_kernel.restype = i32
         L.kvr_last_decode_kernel.argtypes = [vp]
         L.kvr_last_decode_kernel.restype = i32
+        L.kvr_append_sizes.argtypes = [i32, i32, i32, i32, i32, i32, ctypes.POINTER(i32)]
+        L.kvr_append_sizes.restype = i32
+        L.kvr_append.argtypes = [vp, i32, vp, vp, vp, vp, i32, i32, vp, vp, i32, i32, i32, i32, f32, i32, vp, vp, vp, vp, vp, vp]
         L.kvr_measure_pipe_peaks.argtypes = [ctypes.POINTER(ctypes.c_double), vp]
         L.kvr_status_string.argtypes = [i32]
         L.kvr_status_string.restype = ctypes.c_char_p
@@ -357,6 +361,39 @@ def kvr_swap(sk: Sketch, layer: int, Kr, Vr, ret_idx, row_scores, n_recent: int 
                             _stream(stream))
     _check(st, "kvr_swap")
     return n
+
+
+def kvr_append_sizes(n_rows: int, n_recent: int, n_new: int, r_budget: int, c_budget: int, slack: int):
+    """(rows_after, n_recent_after) of kvr_append, from the counts alone."""
+    rec = ctypes.c_int32(0)
+    n = lib().kvr_append_sizes(int(n_rows), int(n_recent), int(n_new), int(r_budget), int(c_budget), int(slack),
+                               ctypes.byref(rec))
+    if n < 0:
+        raise KvrError(KVR_ERR_SHAPE, "kvr_append_sizes")
+    return int(n), int(rec.value)
+
+
+def kvr_append(sk: Sketch, layer: int, Kr, Vr, ret_idx, row_scores, n_recent: int, K_new, V_new, r_budget: int,
+               c_budget: int, slack: int, replace_rate: float = 1.1, max_swaps: int = 1 << 30, stream=None):
+    """kvr_append: Algorithm 3 for the new rows K_new, V_new.  Returns
+    (Kr_out, Vr_out, ret_idx_out, row_scores_out, n_recent_after, n_swapped)."""
+    n_rows, n_new = Kr.shape[-2], K_new.shape[-2]
+    rows_after, rec_after = kvr_append_sizes(n_rows, n_recent, n_new, r_budget, c_budget, slack)
+    lead = tuple(K_new.shape[:-2])
+    Ko = torch.empty(lead + (rows_after, K_new.shape[-1]), dtype=K_new.dtype, device=K_new.device)
+    Vo = torch.empty_like(Ko)
+    ro = torch.empty(lead + (rows_after,), dtype=torch.int32, device=K_new.device)
+    so = torch.empty(lead + (rows_after,), dtype=torch.float32, device=K_new.device)
+    n = torch.zeros(lead, dtype=torch.int32, device=K_new.device)
+    with torch.cuda.device(sk.device):
+        st = lib().kvr_append(sk.handle, layer, _ptr(Kr) if n_rows else None, _ptr(Vr) if n_rows else None,
+                              _ptr(ret_idx) if n_rows else None, _ptr(row_scores) if n_rows else None, n_rows,
+                              int(n_recent), _ptr(K_new) if n_new else None, _ptr(V_new) if n_new else None, n_new,
+                              int(r_budget), int(c_budget), int(slack), float(replace_rate),
+                              int(min(max_swaps, 2 ** 31 - 1)), _ptr(Ko), _ptr(Vo), _ptr(ro), _ptr(so), _ptr(n),
+                              _stream(stream))
+    _check(st, "kvr_append")
+    return Ko, Vo, ro, so, rec_after, n
 
 
 def kvr_compress_host(sk: Sketch, layer: int, K, V, Qobs, budget: int, n_recent: int = 0, stream=None):

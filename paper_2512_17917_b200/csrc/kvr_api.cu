@@ -48,7 +48,7 @@ kvr_status_t ensure(kvr_sketch* sk, void** p, size_t* cur, size_t need) {
 
 void free_all(kvr_sketch* sk) {
     void* ptrs[] = {sk->tok_h, sk->tok_g, sk->tok_pack, sk->full_off, sk->full_list, sk->cells, sk->scores,
-                    sk->cmp_idx, sk->bitmap, sk->dlist, sk->doff, sk->ws_score, sk->ws_decode, sk->tickets, sk->clist, sk->coff, sk->dev_status, sk->ml, sk->ws_demote,
+                    sk->cmp_idx, sk->bitmap, sk->dlist, sk->doff, sk->ws_score, sk->ws_decode, sk->tickets, sk->clist, sk->coff, sk->dev_status, sk->ml, sk->ws_demote, sk->ws_append,
                     sk->st_K, sk->st_V, sk->st_Q, sk->st_Kr, sk->st_Vr, sk->st_ret, sk->st_q1, sk->st_out};
     for (void* p : ptrs)
         if (p) cudaFree(p);
@@ -415,6 +415,80 @@ kvr_status_t kvr_demote(kvr_sketch_t* sk, int32_t layer, const void* Kr, const v
                                row_scores, Kr_out, Vr_out, ret_idx_out, row_scores_out, sk->ws_demote,
                                (cudaStream_t)cuda_stream));
     for (int l = lr.layer0; l < lr.layer0 + lr.n_layers; ++l) { sk->layer_N[l] = new_context; sk->layer_R[l] = budget; }
+    return KVR_OK;
+}
+
+int32_t kvr_append_sizes(int32_t n_rows, int32_t n_recent, int32_t n_new, int32_t r_budget, int32_t c_budget,
+                         int32_t slack, int32_t* n_recent_after) {
+    if (n_rows < 0 || n_recent < 0 || n_recent > n_rows || n_new < 0 || r_budget < 0 || c_budget < 0 || slack < 0) return -1;
+    long long recent = (long long)n_recent + n_new, cand = (long long)n_rows - n_recent;
+    if (recent > (long long)r_budget + slack) { cand += recent - r_budget; recent = r_budget; }
+    if (cand > c_budget) cand = c_budget;
+    if (cand + recent > 0x7FFFFFFF) return -1;
+    if (n_recent_after) *n_recent_after = (int32_t)recent;
+    return (int32_t)(cand + recent);
+}
+
+kvr_status_t kvr_append(kvr_sketch_t* sk, int32_t layer, const void* Kr, const void* Vr, const int32_t* ret_idx,
+                        const float* row_scores, int32_t n_rows, int32_t n_recent, const void* K_new,
+                        const void* V_new, int32_t n_new, int32_t r_budget, int32_t c_budget, int32_t slack,
+                        float replace_rate, int32_t max_swaps, void* Kr_out, void* Vr_out, int32_t* ret_idx_out,
+                        float* row_scores_out, int32_t* n_swapped, void* cuda_stream) {
+    if (!sk || !Kr_out || !Vr_out || !ret_idx_out || !row_scores_out) return KVR_ERR_INVALID_ARG;
+    if (n_rows > 0 && (!Kr || !Vr || !ret_idx || !row_scores)) return KVR_ERR_INVALID_ARG;
+    if (n_new > 0 && (!K_new || !V_new)) return KVR_ERR_INVALID_ARG;
+    if (!aligned16(Kr) || !aligned16(Vr) || !aligned16(K_new) || !aligned16(V_new) || !aligned16(Kr_out) || !aligned16(Vr_out))
+        return KVR_ERR_INVALID_ARG;
+    if (Kr_out == Kr || Vr_out == Vr || ret_idx_out == ret_idx || row_scores_out == row_scores) return KVR_ERR_INVALID_ARG;
+    if (!(replace_rate > 0.f) || isinf(replace_rate) || max_swaps < 0) return KVR_ERR_INVALID_ARG;
+    LayerRange lr;
+    kvr_status_t rc = layer_range(sk, layer, &lr);
+    if (rc != KVR_OK) return rc;
+    int N, R;
+    rc = layer_state(sk, lr, &N, &R);
+    if (rc != KVR_OK) return rc;
+    int32_t recent_after = 0;
+    const int32_t rows_after = kvr_append_sizes(n_rows, n_recent, n_new, r_budget, c_budget, slack, &recent_after);
+    if (rows_after < 0 || n_rows < R) return KVR_ERR_SHAPE;
+    const int rows_cat = n_rows + n_new;
+    const int ctx0 = N + (n_rows - R);                     // every token that arrived since the last compress / overflow step is a row
+    if (ctx0 + n_new > sk->d.max_context) return KVR_ERR_SHAPE;
+    DeviceGuard dg(sk->device);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const bool pops = rows_after < rows_cat;               // known from the counts alone: no device result is waited for
+    if (!pops) {
+        KVR_CUDA(kvr_launch_append_rows(sk, lr.n_inst, Kr, Vr, ret_idx, row_scores, n_rows, K_new, V_new, n_new, ctx0,
+                                        Kr_out, Vr_out, ret_idx_out, row_scores_out, st));
+    } else {
+        // storage + new rows go to a workspace; the overflow step compacts them into the caller's output
+        const size_t row_b = (size_t)KVR_D * 2;
+        const size_t per = (size_t)lr.n_inst * rows_cat;
+        const size_t off_v = (per * row_b + 255) & ~(size_t)255, off_r = off_v + ((per * row_b + 255) & ~(size_t)255);
+        const size_t off_s = off_r + ((per * 4 + 255) & ~(size_t)255), total = off_s + per * 4;
+        rc = ensure(sk, &sk->ws_append, &sk->ws_append_bytes, total);
+        if (rc != KVR_OK) return rc;
+        rc = ensure(sk, &sk->ws_demote, &sk->ws_demote_bytes, kvr_demote_ws_bytes(lr.n_inst, rows_cat));
+        if (rc != KVR_OK) return rc;
+        char* w = (char*)sk->ws_append;
+        KVR_CUDA(kvr_launch_append_rows(sk, lr.n_inst, Kr, Vr, ret_idx, row_scores, n_rows, K_new, V_new, n_new, ctx0,
+                                        w, w + off_v, (int32_t*)(w + off_r), (float*)(w + off_s), st));
+        sk->chain = false;
+        for (int l = lr.layer0; l < lr.layer0 + lr.n_layers; ++l) sk->layer_N[l] = sk->layer_R[l] = -1;
+        KVR_CUDA(kvr_launch_demote(sk, lr.inst0, lr.n_inst, rows_cat, ctx0 + n_new, rows_after, recent_after, w, w + off_v,
+                                   (const int32_t*)(w + off_r), (const float*)(w + off_s), Kr_out, Vr_out, ret_idx_out,
+                                   row_scores_out, sk->ws_demote, st));
+        N = ctx0 + n_new;
+        R = rows_after;
+        for (int l = lr.layer0; l < lr.layer0 + lr.n_layers; ++l) { sk->layer_N[l] = N; sk->layer_R[l] = R; }
+    }
+    // the swap loop runs on every call (Algorithm 3), on the device, over what the steps above left
+    if (rows_after - recent_after > 0 && N - R > 0 && max_swaps > 0) {
+        sk->chain = false;
+        KVR_CUDA(kvr_launch_swap(sk, lr.inst0, lr.n_inst, N, N - R, Kr_out, Vr_out, ret_idx_out, row_scores_out, rows_after,
+                                 recent_after, replace_rate, max_swaps, n_swapped, st));
+    } else if (n_swapped) {
+        KVR_CUDA(cudaMemsetAsync(n_swapped, 0, sizeof(int32_t) * lr.n_inst, st));
+    }
     return KVR_OK;
 }
 

@@ -75,6 +75,7 @@ struct kvr_sketch {
     float* ml;                                // [n_inst][G][2] softmax reference maximum (log2 units) and sum of
                                               // the last decode of each head-instance (for score accumulation)
     void* ws_demote; size_t ws_demote_bytes;  // positions / membership of the overflow step
+    void* ws_append; size_t ws_append_bytes;  // storage + new rows before the overflow step of kvr_append
 
     // ---- host-buffer path (allocated on first use) ----
     void* st_K; void* st_V; void* st_Q; size_t st_k_bytes, st_v_bytes, st_q_bytes;
@@ -170,6 +171,10 @@ cudaError_t kvr_launch_demote(kvr_sketch* sk, int inst0, int n_inst, int rows, i
                               const void* Kr, const void* Vr, const int32_t* ret_idx, const float* row_scores,
                               void* Kr_out, void* Vr_out, int32_t* ret_out, float* scores_out, void* ws,
                               cudaStream_t st);
+
+cudaError_t kvr_launch_append_rows(kvr_sketch* sk, int n_inst, const void* Kr, const void* Vr, const int32_t* ret,
+                                   const float* rs, int rows, const void* Kn, const void* Vn, int n_new, int ctx0,
+                                   void* Ko, void* Vo, int32_t* ro, float* so, cudaStream_t st);
 
 size_t kvr_decode_ws_bytes(int n_inst, int n_splits, int G);
 int kvr_decode_pick_splits(const kvr_sketch* sk, int n_inst, int N, int R);

@@ -287,7 +287,43 @@ cmp_from_bitmap_kernel(const uint32_t* __restrict__ bitmap_all, int bitmap_words
     }
 }
 
+// Storage of a head-instance followed by the newly arrived rows (Algorithm 3 pushes new tokens to the
+// Recent part, which is the tail of the storage): rows, token indices (the new tokens are numbered
+// ctx0, ctx0 + 1, ...) and row scores (a new token has received no attention yet: 0).
+__global__ void append_rows_kernel(const uint4* __restrict__ Kr, const uint4* __restrict__ Vr,
+                                   const int32_t* __restrict__ ret, const float* __restrict__ rs, int rows,
+                                   const uint4* __restrict__ Kn, const uint4* __restrict__ Vn, int n_new, int ctx0,
+                                   uint4* __restrict__ Ko, uint4* __restrict__ Vo, int32_t* __restrict__ ro,
+                                   float* __restrict__ so) {
+    const int u = blockIdx.y, total = rows + n_new;
+    constexpr int RV = KVR_D * 2 / 16;                        // 16-byte pieces of a 16-bit row
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total * RV; i += gridDim.x * blockDim.x) {
+        const int row = i / RV, c = i - row * RV;
+        const bool old = row < rows;
+        const size_t src = old ? ((size_t)u * rows + row) * RV + c : ((size_t)u * n_new + (row - rows)) * RV + c;
+        Ko[((size_t)u * total + row) * RV + c] = old ? Kr[src] : Kn[src];
+        Vo[((size_t)u * total + row) * RV + c] = old ? Vr[src] : Vn[src];
+    }
+    for (int row = blockIdx.x * blockDim.x + threadIdx.x; row < total; row += gridDim.x * blockDim.x) {
+        ro[(size_t)u * total + row] = row < rows ? ret[(size_t)u * rows + row] : ctx0 + (row - rows);
+        so[(size_t)u * total + row] = row < rows ? rs[(size_t)u * rows + row] : 0.f;
+    }
+}
+
 }  // namespace
+
+cudaError_t kvr_launch_append_rows(kvr_sketch* sk, int n_inst, const void* Kr, const void* Vr, const int32_t* ret,
+                                   const float* rs, int rows, const void* Kn, const void* Vn, int n_new, int ctx0,
+                                   void* Ko, void* Vo, int32_t* ro, float* so, cudaStream_t st) {
+    if (rows + n_new <= 0 || n_inst <= 0) return cudaSuccess;
+    const int total = rows + n_new;
+    int gx = (total * 16 + 255) / 256;
+    if (gx > 64) gx = 64;
+    append_rows_kernel<<<dim3(gx, n_inst), 256, 0, st>>>((const uint4*)Kr, (const uint4*)Vr, ret, rs, rows, (const uint4*)Kn,
+                                                         (const uint4*)Vn, n_new, ctx0, (uint4*)Ko, (uint4*)Vo, ro, so);
+    sk->launches += 1;
+    return cudaGetLastError();
+}
 
 cudaError_t kvr_launch_row_mass(kvr_sketch* sk, int inst0, int n_inst, int rows, const void* q, const void* Kr,
                                 float scale, float* acc, cudaStream_t st) {

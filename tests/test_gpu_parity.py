@@ -351,6 +351,88 @@ def test_swap_loop_and_vague_scores(which, dtype, rate):
     kvr.kvr_sketch_destroy(sk)
 
 
+@pytest.mark.parametrize("which,dtype", [("staged", F16), ("split", BF16)])
+def test_append_runs_algorithm_3_over_several_slack_periods(which, dtype):
+    """kvr_append against the oracle's compress_stream: a generation loop of decode, score
+    accumulation (stored rows and vague tokens) and one kvr_append per step, through more than three
+    Slack periods.  Which rows stay and which tokens are swapped are integer decisions taken in fp32
+    from the scores the kernels accumulated, so row indices, row scores and per-token scores are
+    compared exactly; cells and rows within the tolerance; the decode of every step is compared with
+    the oracle on the storage of that step."""
+    B, H, Hq, N, R, b, n_rec0 = 1, 2, 8, 1000, 120, 30, 10
+    G = Hq // H
+    r_budget, c_budget, slack = 10, 110, 6
+    n_inst = B * H
+    seeds = synth.hash_seeds(4711)
+    steps = [3, 1, 2, 4, 1, 3, 2, 2, 4, 1, 3, 2]
+    total = N + sum(steps)
+    K, V, Q, q = make_case(4712, B, H, Hq, total, 8, dtype, 1)
+    dev = "cuda"
+    sk = kvr.kvr_sketch_create(b=b, batch=B, n_layers=1, n_kv_heads=H, n_q_heads=Hq, max_context=total, kv_dtype=dtype,
+                               hash_seeds=seeds)
+    kvr.kvr_sketch_set_decode_kernel(sk, kvr.KVR_DECODE_SPLIT if which == "split" else kvr.KVR_DECODE_STAGED)
+    Kall, Vall = inst_major(K[0]), inst_major(V[0])
+    Kr, Vr, ret = kvr.kvr_compress(sk, 0, K[0, :, :, :N].contiguous().to(dev), V[0, :, :, :N].contiguous().to(dev),
+                                   Q[0].to(dev), R, n_rec0)
+    cmp0 = kvr.kvr_get_assignment(sk, 0)[0].reshape(n_inst, -1).cpu().numpy()
+    s0 = kvr.kvr_get_scores(sk, 0).reshape(n_inst, -1)
+    acc = torch.gather(s0, 1, ret.reshape(n_inst, -1).long()).reshape(B, H, R).contiguous()
+    # oracle state per head-instance
+    o_cells = list(orc.insert(Kall[:, :N], Vall[:, :N], cmp0, seeds, b))
+    o_Kr, o_Vr = list(inst_major(Kr).astype(np.float64)), list(inst_major(Vr).astype(np.float64))
+    o_ret = list(ret.reshape(n_inst, -1).cpu().numpy())
+    n_recent, ctx, drops, swaps = n_rec0, N, 0, 0
+    rounder = lambda x: torch.from_numpy(np.asarray(x, np.float64)).to(dtype).double().numpy()
+    ulp = 2.0 ** -11 if dtype == F16 else 2.0 ** -8
+    for it, n_new in enumerate(steps):
+        # ---- decode over the current storage, then the attention mass goes to the scores
+        qd = synth.make_decode_q(5000 + it, B, Hq, 128, dtype, dev)
+        out = kvr.kvr_decode_attention(sk, 0, qd, Kr, Vr, ret)
+        kvr.kvr_accumulate_scores(sk, 0, qd, Kr, acc)
+        kvr.kvr_accumulate_vague_scores(sk, 0, qd)
+        qo = dec_to_inst(qd, H)
+        want = orc.decode(qo, np.stack(o_Kr), np.stack(o_Vr), np.stack(o_ret), np.stack(o_cells), ctx, seeds)
+        assert np.abs(out.reshape(n_inst, G, 128).cpu().numpy() - want).max() <= TOL
+        tok_g = kvr.kvr_get_scores(sk, 0).reshape(n_inst, -1).cpu().numpy()       # [n_inst, context of the last overflow step]
+        acc_np = acc.reshape(n_inst, -1).cpu().numpy()
+        # ---- Algorithm 3 for the new tokens
+        Kn, Vn = K[0, :, :, ctx:ctx + n_new].contiguous().to(dev), V[0, :, :, ctx:ctx + n_new].contiguous().to(dev)
+        before = n_recent + n_new
+        Kr, Vr, ret, acc, n_recent_g, n_sw = kvr.kvr_append(sk, 0, Kr, Vr, ret, acc, n_recent, Kn, Vn, r_budget, c_budget,
+                                                            slack, 1.1, 20)
+        assert kvr.kvr_sketch_device_status(sk) == 0
+        n_sw = n_sw.reshape(n_inst).cpu().numpy()
+        ret_g, acc_g = ret.reshape(n_inst, -1).cpu().numpy(), acc.reshape(n_inst, -1).cpu().numpy()
+        cells_g = kvr.kvr_get_cells(sk, 0).reshape(n_inst, 2, 3, b, 128).cpu().numpy().transpose(0, 2, 3, 1, 4)
+        tok_after = kvr.kvr_get_scores(sk, 0).reshape(n_inst, -1).cpu().numpy()
+        for u in range(n_inst):
+            # the oracle steps from its own storage, with the scores the kernels accumulated
+            tok_u = np.concatenate([tok_g[u], np.zeros(ctx + n_new - tok_g.shape[1], np.float32)])   # tokens beyond are rows
+            Ko, Vo, ro, so, rec_o, to, co, n = orc.compress_stream(
+                o_Kr[u], o_Vr[u], o_ret[u], acc_np[u], n_recent, tok_u, o_cells[u], Kall[u, ctx:ctx + n_new],
+                Vall[u, ctx:ctx + n_new], np.arange(ctx, ctx + n_new, dtype=np.int32), r_budget, c_budget, slack, 1.1, 20,
+                seeds, round_rows=rounder)
+            assert rec_o == n_recent_g and n == n_sw[u]
+            assert (ret_g[u] == ro).all() and (acc_g[u] == so).all()
+            vague = np.setdiff1d(np.arange(ctx + n_new), ro)
+            assert (tok_after[u, vague] == to[vague]).all()
+            assert np.abs(cells_g[u] - co).max() <= TOL
+            dk, dv = np.abs(inst_major(Kr)[u] - Ko), np.abs(inst_major(Vr)[u] - Vo)
+            assert (dk <= TOL + 2 * ulp * np.abs(Ko)).all() and (dv <= TOL + 2 * ulp * np.abs(Vo)).all()
+            # carry the GPU's rows on (a revived row is rounded to the cache type on both sides)
+            o_Kr[u], o_Vr[u], o_ret[u], o_cells[u] = inst_major(Kr)[u].astype(np.float64), inst_major(Vr)[u].astype(np.float64), ro, co
+            swaps += n
+        drops += int(n_recent_g < before)
+        n_recent, ctx = n_recent_g, ctx + n_new
+    assert drops >= 3 and swaps > 0
+    # ---- one more decode over the final storage
+    qd = synth.make_decode_q(5999, B, Hq, 128, dtype, dev)
+    out = kvr.kvr_decode_attention(sk, 0, qd, Kr, Vr, ret)
+    want = orc.decode(dec_to_inst(qd, H), np.stack(o_Kr), np.stack(o_Vr), np.stack(o_ret), np.stack(o_cells), ctx, seeds)
+    assert np.abs(out.reshape(n_inst, G, 128).cpu().numpy() - want).max() <= TOL
+    kvr.kvr_sketch_destroy(sk)
+
+
 def test_per_layer_budgets_in_one_handle():
     """Budgets that differ from layer to layer (kvr_layer_budgets from per-layer weights): every layer
     of one handle is compressed with its own budget and decoded; selection, cells and outputs against
