@@ -188,6 +188,25 @@ def decode(q, Kr, Vr, ret_idx, cells, N: int, seeds, scale: float | None = None,
     return out
 
 
+def decode_mq(q, Kr, Vr, ret_idx, cells, N: int, seeds, causal: bool = True, scale: float | None = None,
+              mix: bool = True, combine: str = "median") -> np.ndarray:
+    """Several queries per head over the same storage (speculative / chunked decoding): the cache is
+    rebuilt by Algorithm 4 and every query attends to it as in `decode`.  q [n_inst, G, Qn, D].
+    causal: the last Qn rows of the storage are the queries' own tokens (token indices N - Qn .. N - 1,
+    in order); query t sees the cache up to and including its own token, i.e. the first
+    rows - Qn + t + 1 rows and the first N - Qn + t + 1 tokens.  Not causal: every query sees all of it.
+    out float64 [n_inst, G, Qn, D]."""
+    q = _f32(q)
+    n_inst, G, Qn, D = q.shape
+    rows = _i32(ret_idx).shape[1]
+    out = np.empty((n_inst, G, Qn, D), np.float64)
+    for t in range(Qn):
+        cut = Qn - 1 - t if causal else 0
+        out[:, :, t] = decode(q[:, :, t], _f32(Kr)[:, :rows - cut], _f32(Vr)[:, :rows - cut], _i32(ret_idx)[:, :rows - cut],
+                              cells, N - cut, seeds, scale, mix, combine)
+    return out
+
+
 def decode_mass(q, Kr, Vr, ret_idx, cells, N: int, seeds, scale: float | None = None,
                 mix: bool = True) -> np.ndarray:
     """Attention mass of every one of the N tokens in one decode step (sum over the G query heads

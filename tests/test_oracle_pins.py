@@ -510,6 +510,66 @@ def test_swap_rate_and_limit():
     np.testing.assert_allclose(out[5], step[0], rtol=0, atol=1e-12)
 
 
+def _sdpa_causal_tail(q, K, V, Qn, causal):
+    """torch fp64 attention of Qn queries per head over N tokens; with `causal`, query t is token
+    N - Qn + t and sees the tokens up to itself (mask written out)."""
+    n_inst, G, _, D = q.shape
+    N = K.shape[1]
+    qt, Kt, Vt = (torch.from_numpy(np.asarray(x, np.float64)) for x in (q, K, V))
+    logits = torch.einsum("ugtd,ujd->ugtj", qt, Kt) / np.sqrt(D)
+    if causal:
+        j = torch.arange(N)[None, :]
+        t = torch.arange(Qn)[:, None]
+        logits = logits.masked_fill((j > N - Qn + t)[None, None], float("-inf"))
+    return torch.einsum("ugtj,ujd->ugtd", torch.softmax(logits, dim=-1), Vt).numpy()
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_decode_mq_at_full_budget_is_masked_textbook_attention(causal):
+    """Nothing compressed: Qn queries per head against a library softmax attention with the causal
+    mask among the queries' own tokens written out."""
+    n_inst, G, Qn, N, D = 2, 3, 5, 37, 8
+    q = _rand((n_inst, G, Qn, D), 800)
+    K, V = _rand((n_inst, N, D), 801), _rand((n_inst, N, D), 802)
+    seeds = synth.hash_seeds(803)
+    ret = np.arange(N, dtype=np.int32)[None].repeat(n_inst, 0)
+    cells = np.zeros((n_inst, 3, 4, 2, D))
+    got = orc.decode_mq(q, K, V, ret, cells, N, seeds, causal=causal)
+    np.testing.assert_allclose(got, _sdpa_causal_tail(q, K, V, Qn, causal), rtol=1e-10, atol=1e-12)
+
+
+def test_decode_mq_under_injective_hashing_and_against_single_query_decode():
+    """Partial budget with one cell per token: the rebuilt cache is the original one, so the result is
+    masked attention over the original K, V; one query per head is `decode`; without the mask every
+    query is `decode` over the whole storage; the last query of the causal form sees everything."""
+    n_inst, G, Qn, N0, D = 2, 2, 4, 30, 8
+    N = N0 + Qn
+    q = _rand((n_inst, G, Qn, D), 810)
+    K, V = _rand((n_inst, N, D), 811), _rand((n_inst, N, D), 812)
+    Qobs = _rand((n_inst, 6, D), 813)
+    seeds = synth.injective_seeds()
+    c = orc.compress(Qobs, K[:, :N0], V[:, :N0], R=9, n_recent=2, seeds=seeds, b=N, mix=False)
+    new = np.arange(N0, N, dtype=np.int32)[None].repeat(n_inst, 0)
+    Kr, Vr = np.concatenate([c["Kr"], K[:, N0:]], axis=1), np.concatenate([c["Vr"], V[:, N0:]], axis=1)
+    ret = np.concatenate([c["ret_idx"], new], axis=1)
+    got = orc.decode_mq(q, Kr, Vr, ret, c["cells"], N, seeds, causal=True, mix=False)
+    np.testing.assert_allclose(got, _sdpa_causal_tail(q, K, V, Qn, True), rtol=1e-9, atol=1e-11)
+    free = orc.decode_mq(q, Kr, Vr, ret, c["cells"], N, seeds, causal=False, mix=False)
+    for t in range(Qn):
+        np.testing.assert_allclose(free[:, :, t], orc.decode(q[:, :, t], Kr, Vr, ret, c["cells"], N, seeds, mix=False), rtol=0, atol=0)
+    np.testing.assert_allclose(got[:, :, Qn - 1], free[:, :, Qn - 1], rtol=0, atol=0)
+    one = orc.decode_mq(q[:, :, :1], Kr, Vr, ret, c["cells"], N, seeds, causal=False, mix=False)
+    np.testing.assert_allclose(one[:, :, 0], orc.decode(q[:, :, 0], Kr, Vr, ret, c["cells"], N, seeds, mix=False), rtol=0, atol=0)
+    # with collisions (ordinary hashing) the mask still only hides the later queries' tokens
+    seeds2 = synth.hash_seeds(814)
+    c2 = orc.compress(Qobs, K[:, :N0], V[:, :N0], R=9, n_recent=2, seeds=seeds2, b=3)
+    Kr2, Vr2 = np.concatenate([c2["Kr"], K[:, N0:]], axis=1), np.concatenate([c2["Vr"], V[:, N0:]], axis=1)
+    ret2 = np.concatenate([c2["ret_idx"], new], axis=1)
+    mq = orc.decode_mq(q, Kr2, Vr2, ret2, c2["cells"], N, seeds2, causal=True)
+    first = orc.decode(q[:, :, 0], Kr2[:, :9 + 1], Vr2[:, :9 + 1], ret2[:, :9 + 1], c2["cells"], N0 + 1, seeds2)
+    np.testing.assert_allclose(mq[:, :, 0], first, rtol=0, atol=0)
+
+
 def _stream_case(seed, N=40, n_total=64, D=8, b=5, R=14, n_recent=4, injective=False):
     Q = _rand((1, 8, D), seed)
     K, V = _rand((1, n_total, D), seed + 1), _rand((1, n_total, D), seed + 2)
