@@ -417,6 +417,87 @@ def run_stream(args, w):
     return res
 
 
+# ------------------------------------------------------------------- several queries per head
+def run_mq(args, w):
+    """--queries Qn: decode attention for Qn queries per head per call (kvr_decode_attention_mq) over the
+    compressed cache of the workload, one call per layer, all layers and decode steps replayed from a
+    CUDA graph.  One JSON line: query tokens per second, the time per layer call, the same bytes-based
+    roofline as the single-query line (the cache is read once per call whatever Qn is), and the time
+    of Qn single-query calls beside it."""
+    import paper_2512_17917_b200 as kvr
+
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    L, B, H, Hq, D, N, R, Qn = w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, w.head_dim, w.context, w.budget, args.queries
+    S = max(1, min(w.decode_steps, 16))
+    dt = w.torch_dtype
+    sk = kvr.kvr_sketch_create(b=w.b, batch=B, n_layers=L, n_kv_heads=H, n_q_heads=Hq, max_context=N, kv_dtype=dt,
+                               hash_seeds=synth.hash_seeds(w.seed + 3), device=dev)
+    st = []
+    for layer in range(L):
+        K, V, Q = synth.layer_inputs(w, layer, dev)
+        st.append(kvr.kvr_compress(sk, layer, K, V, Q, R, w.n_recent))
+        del K, V, Q
+    gen = torch.Generator(device=dev).manual_seed(w.seed + 77)
+    qm = torch.randn((S, L, B, Hq, Qn, D), generator=gen, device=dev).to(dt)
+    out = torch.empty((L, B, Hq, Qn, D), dtype=torch.float32, device=dev)
+    out1 = torch.empty((L, B, Hq, D), dtype=torch.float32, device=dev)
+
+    def graph_of(fn):
+        fn()
+        torch.cuda.synchronize()
+        g, side = torch.cuda.CUDAGraph(), torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                fn()
+        torch.cuda.synchronize()
+        return g
+
+    def mq_all():
+        for s in range(S):
+            for layer in range(L):
+                kvr.kvr_decode_attention_mq(sk, layer, qm[s, layer], *st[layer], causal=False, out=out[layer])
+
+    def single_all():
+        for s in range(S):
+            for layer in range(L):
+                kvr.kvr_decode_attention(sk, layer, qm[s, layer, :, :, 0].contiguous(), *st[layer], out=out1[layer])
+
+    def timed(g, reps):
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    ms_mq = timed(graph_of(mq_all), max(1, args.steps))
+    ms_1 = timed(graph_of(single_all), max(1, args.steps))
+    assert kvr.kvr_sketch_device_status(sk) == 0 and torch.isfinite(out).all()
+    peak, peak_kind = measured_peaks()
+    call_us = ms_mq * 1e3 / (S * L)
+    bytes_call = decode_bytes_per_launch(w, B * H) + B * Hq * Qn * D * 6
+    res = {"metric": METRIC, "value": round(B * Qn * S / (ms_mq * 1e-3), 2), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+           "warmup": 3, "ms_per_step": round(ms_mq, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+           "dtype": "f32 accumulate, f16 hi+lo operands", "data": "synthetic",
+           "config": dict(config_of(w), queries_per_head=Qn, decode_steps_per_step=S, launch="per_layer_cuda_graph"),
+           "decode_kernel": "decode_mq_kernel", "layer_call_us": round(call_us, 2),
+           "launches_per_layer_call": (Hq // H * Qn + 15) // 16,
+           "roofline": {"kernel": "decode_mq_kernel", "bound": "hbm", "achieved": round(bytes_call / (call_us * 1e-6) / 1e9, 1),
+                        "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                        "frac": round(bytes_call / (call_us * 1e-6) / 1e9 / peak, 4), "bytes_per_launch": bytes_call,
+                        "avg_launch_us": round(call_us, 2), "traffic": None},
+           "single_query": {"layer_call_us": round(ms_1 * 1e3 / (S * L), 2),
+                            "speedup_per_query": round(Qn * ms_1 / ms_mq, 2)},
+           "gpu_launches": int(S * L * ((Hq // H * Qn + 15) // 16))}
+    kvr.kvr_sketch_destroy(sk)
+    return res
+
+
 # ----------------------------------------------------------------------------- the CPU oracle
 def oracle_sample(w, n_sample: int, decode_steps: int, inputs=None, combine: str = "median"):
     """Time the oracle, as it stands, on n_sample head-instances of layer 0: one compress and
@@ -488,6 +569,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="kvr", choices=["kvr", "reference"])
     ap.add_argument("--stream", type=int, default=0, help="time T generation steps with Algorithm 3 (kvr_append) instead")
+    ap.add_argument("--queries", type=int, default=0, help="time decode attention with this many queries per head per call instead")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling a small case)")
@@ -536,6 +618,9 @@ def main():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback of the hot path)")
     if args.stream > 0:
         print(json.dumps(run_stream(args, w)), flush=True)
+        return
+    if args.queries > 0:
+        print(json.dumps(run_mq(args, w)), flush=True)
         return
     if args.warmup < 3:
         args.warmup = 3

@@ -139,6 +139,26 @@ kvr_status_t kvr_decode_attention(kvr_sketch_t* sk, int32_t layer, const void* q
                                   const void* Vr, const int32_t* ret_idx, int32_t n_retained,
                                   float softmax_scale, float* out, void* cuda_stream);
 
+/* Several queries per head over the same storage (speculative decoding, chunked prefill): the cache
+ * is rebuilt once per tile of tokens (Algorithm 4, Algorithm 2 for the vague tokens) and serves all
+ * queries, so the reconstruction cost of the Calculation Phase is shared (paper, Throughput Analysis:
+ * the rebuild comes first, the attention after it).
+ *   q    device [batch, n_q_heads, n_queries, head_dim] (kv_dtype)
+ *   out  device [batch, n_q_heads, n_queries, head_dim] float32
+ *   Kr, Vr, ret_idx, n_retained as in kvr_decode_attention (rows appended after the compress included).
+ *   causal = 1: the last n_queries rows of the storage are the queries' own tokens, in order; query t
+ *               sees the cache up to and including its own token (rows < n_retained - n_queries + t + 1).
+ *   causal = 0: every query sees the whole storage.
+ * The two contractions run on the tensor cores on 16-bit halves of the reconstructed vectors
+ * (x = hi + lo, 22 significant bits; fp32 accumulation): reconstructed values beyond the 16-bit float
+ * range (65504) are not supported.  Needs a handle with a class grid (as the staged decode kernel:
+ * at most 4 query heads per kv head, b up to about 540): KVR_ERR_UNSUPPORTED otherwise.
+ * Errors: INVALID_ARG, SHAPE, STATE, UNSUPPORTED, ALLOC, CUDA. */
+kvr_status_t kvr_decode_attention_mq(kvr_sketch_t* sk, int32_t layer, const void* q, const void* Kr,
+                                     const void* Vr, const int32_t* ret_idx, int32_t n_retained,
+                                     int32_t n_queries, int32_t causal, float softmax_scale, float* out,
+                                     void* cuda_stream);
+
 /* kvr_decode_attention without any allocation (the paper has no counterpart: this is a property
  * of the library, not of the method).  For callers that cannot allocate device memory when they
  * decode -- a serving process whose own pool already holds all free device memory, so that a

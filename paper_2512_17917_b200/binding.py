@@ -32,7 +32,7 @@ EXPORTS = (
     "kvr_sketch_set_decode_kernel", "kvr_last_decode_kernel", "kvr_sketch_device_status",
     "kvr_accumulate_scores", "kvr_demote", "kvr_sketch_set_score_kernel", "kvr_last_score_kernel",
     "kvr_accumulate_vague_scores", "kvr_swap", "kvr_sketch_set_obs_window_causal", "kvr_paper_storage_split", "kvr_layer_budgets", "kvr_sketch_set_combine",
-    "kvr_measure_pipe_peaks", "kvr_append", "kvr_append_sizes",
+    "kvr_measure_pipe_peaks", "kvr_append", "kvr_append_sizes", "kvr_decode_attention_mq",
 )
 
 
@@ -95,6 +95,7 @@ def lib() -> ctypes.CDLL:
         L.kvr_last_score_kernel.restype = i32
         L.kvr_last_decode_kernel.argtypes = [vp]
         L.kvr_last_decode_kernel.restype = i32
+        L.kvr_decode_attention_mq.argtypes = [vp, i32, vp, vp, vp, vp, i32, i32, i32, f32, vp, vp]
         L.kvr_append_sizes.argtypes = [i32, i32, i32, i32, i32, i32, ctypes.POINTER(i32)]
         L.kvr_append_sizes.restype = i32
         L.kvr_append.argtypes = [vp, i32, vp, vp, vp, vp, i32, i32, vp, vp, i32, i32, i32, i32, f32, i32, vp, vp, vp, vp, vp, vp]
@@ -291,6 +292,24 @@ def kvr_decode_attention(sk: Sketch, layer: int, q, Kr, Vr, ret_idx, *, softmax_
                                     _ptr(ret_idx) if R else None, R, float(softmax_scale), _ptr(out),
                                     _stream(stream))
     _check(st, "kvr_decode_attention")
+    return out
+
+
+def kvr_decode_attention_mq(sk: Sketch, layer: int, q, Kr, Vr, ret_idx, *, causal: bool = True, softmax_scale: float = 0.0,
+                            out=None, stream=None):
+    """kvr_decode_attention_mq: q [.., n_q_heads, n_queries, head_dim] -> out of the same shape (float32)."""
+    d = sk.desc
+    lead = _lead(sk, layer)
+    Qn = q.shape[-2]
+    assert tuple(q.shape) == lead + (d.n_q_heads, Qn, d.head_dim) and q.dtype == sk.torch_dtype, "q shape/dtype"
+    R = Kr.shape[-2]
+    if out is None:
+        out = torch.empty(lead + (d.n_q_heads, Qn, d.head_dim), dtype=torch.float32, device=q.device)
+    with torch.cuda.device(sk.device):
+        st = lib().kvr_decode_attention_mq(sk.handle, layer, _ptr(q), _ptr(Kr) if R else None, _ptr(Vr) if R else None,
+                                           _ptr(ret_idx) if R else None, R, int(Qn), int(bool(causal)),
+                                           float(softmax_scale), _ptr(out), _stream(stream))
+    _check(st, "kvr_decode_attention_mq")
     return out
 
 

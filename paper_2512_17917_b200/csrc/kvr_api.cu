@@ -334,6 +334,35 @@ kvr_status_t kvr_decode_attention(kvr_sketch_t* sk, int32_t layer, const void* q
     return decode_impl(sk, lr, N, R, n_retained, q, Kr, Vr, softmax_scale, out, (cudaStream_t)cuda_stream);
 }
 
+kvr_status_t kvr_decode_attention_mq(kvr_sketch_t* sk, int32_t layer, const void* q, const void* Kr, const void* Vr,
+                                     const int32_t* ret_idx, int32_t n_retained, int32_t n_queries, int32_t causal,
+                                     float softmax_scale, float* out, void* cuda_stream) {
+    (void)ret_idx;
+    if (!sk || !q || !out) return KVR_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(Kr) || !aligned16(Vr) || !aligned16(out)) return KVR_ERR_INVALID_ARG;
+    if (!(softmax_scale >= 0.f) || isinf(softmax_scale) || (causal != 0 && causal != 1)) return KVR_ERR_INVALID_ARG;
+    LayerRange lr;
+    kvr_status_t rc = layer_range(sk, layer, &lr);
+    if (rc != KVR_OK) return rc;
+    int N, R;
+    rc = layer_state(sk, lr, &N, &R);
+    if (rc != KVR_OK) return rc;
+    if (n_queries < 1 || n_queries > 4096 || n_retained < R) return KVR_ERR_SHAPE;
+    if (causal && n_retained < n_queries) return KVR_ERR_SHAPE;     // the last rows are the queries' own tokens
+    if (n_retained > 0 && (!Kr || !Vr)) return KVR_ERR_INVALID_ARG;
+    int S, lcap;
+    size_t smem;
+    if (!kvr_decode_mq_plan(sk, lr.n_inst, N, R, &S, &lcap, &smem)) return KVR_ERR_UNSUPPORTED;
+    DeviceGuard dg(sk->device);
+    rc = ensure(sk, &sk->ws_decode, &sk->ws_decode_bytes, kvr_decode_mq_ws_bytes(lr.n_inst, sk->C * sk->C * S));
+    if (rc != KVR_OK) return rc;
+    if (softmax_scale == 0.f) softmax_scale = (float)(1.0 / sqrt((double)sk->d.head_dim));
+    sk->chain = false;
+    KVR_CUDA(kvr_launch_decode_mq(sk, lr.inst0, lr.n_inst, n_retained, q, Kr, Vr, n_queries, causal, softmax_scale, out, S,
+                                  lcap, smem, (float*)sk->ws_decode, (cudaStream_t)cuda_stream));
+    return KVR_OK;
+}
+
 kvr_status_t kvr_accumulate_scores(kvr_sketch_t* sk, int32_t layer, const void* q, const void* Kr, int32_t n_rows,
                                    float softmax_scale, float* score_acc, void* cuda_stream) {
     if (!sk || !q || !score_acc) return KVR_ERR_INVALID_ARG;

@@ -176,6 +176,13 @@ cudaError_t kvr_launch_append_rows(kvr_sketch* sk, int n_inst, const void* Kr, c
                                    const float* rs, int rows, const void* Kn, const void* Vn, int n_new, int ctx0,
                                    void* Ko, void* Vo, int32_t* ro, float* so, cudaStream_t st);
 
+// several queries per head (kvr_decode_mq.cu)
+bool kvr_decode_mq_plan(const kvr_sketch* sk, int n_inst, int N, int R, int* S_out, int* lcap_out, size_t* smem_out);
+size_t kvr_decode_mq_ws_bytes(int n_inst, int records);
+cudaError_t kvr_launch_decode_mq(kvr_sketch* sk, int inst0, int n_inst, int rows, const void* q, const void* Kr, const void* Vr,
+                                 int n_queries, int causal, float scale, float* out, int S, int lcap, size_t smem, float* part,
+                                 cudaStream_t st);
+
 size_t kvr_decode_ws_bytes(int n_inst, int n_splits, int G);
 int kvr_decode_pick_splits(const kvr_sketch* sk, int n_inst, int N, int R);
 

@@ -433,6 +433,66 @@ def test_append_runs_algorithm_3_over_several_slack_periods(which, dtype):
     kvr.kvr_sketch_destroy(sk)
 
 
+@pytest.mark.parametrize("Qn,dtype,causal,b,N0,R", [
+    (1, F16, True, 20, 1200, 150),          # one query: the single-query result
+    (4, F16, True, 20, 1200, 150),          # 16 query rows = one launch
+    (4, BF16, False, 20, 1200, 150),
+    (16, F16, True, 200, 5000, 900),        # 64 query rows = four launches; 4 x 4 classes
+    (16, BF16, True, 20, 700, 100),
+    (3, F16, True, 37, 900, 0),             # nothing retained but the queries' own tokens; 12 rows (padded to 16)
+])
+def test_multi_query_decode_against_the_oracle(Qn, dtype, causal, b, N0, R):
+    """kvr_decode_attention_mq: Qn queries per head over the compressed cache plus the queries' own
+    tokens as appended exact rows, against the oracle's decode_mq (cache rebuilt, every query with its
+    own mask), within the tolerance; Qn = 1 also against the single-query entry point."""
+    B, H, Hq = 1, 2, 8
+    G = Hq // H
+    n_inst = B * H
+    seeds = synth.hash_seeds(3300 + Qn)
+    K, V, Q, _ = make_case(3301 + Qn, B, H, Hq, N0 + Qn, 8, dtype, 1)
+    dev = "cuda"
+    sk = kvr.kvr_sketch_create(b=b, batch=B, n_layers=1, n_kv_heads=H, n_q_heads=Hq, max_context=N0 + Qn, kv_dtype=dtype,
+                               hash_seeds=seeds)
+    Kr, Vr, ret = kvr.kvr_compress(sk, 0, K[0, :, :, :N0].contiguous().to(dev), V[0, :, :, :N0].contiguous().to(dev),
+                                   Q[0].to(dev), R, 0)
+    cmp0 = kvr.kvr_get_assignment(sk, 0)[0].reshape(n_inst, -1).cpu().numpy()
+    cells_o = orc.insert(inst_major(K[0])[:, :N0], inst_major(V[0])[:, :N0], cmp0, seeds, b)
+    Kr2 = torch.cat([Kr, K[0, :, :, N0:].to(dev)], dim=2).contiguous()
+    Vr2 = torch.cat([Vr, V[0, :, :, N0:].to(dev)], dim=2).contiguous()
+    ret2 = torch.cat([ret, torch.arange(N0, N0 + Qn, dtype=torch.int32, device=dev).expand(B, H, Qn)], dim=2).contiguous()
+    gen = torch.Generator().manual_seed(3302 + Qn)
+    qm = torch.randn((B, Hq, Qn, 128), generator=gen).to(dtype)
+    out = kvr.kvr_decode_attention_mq(sk, 0, qm.to(dev), Kr2, Vr2, ret2, causal=causal)
+    torch.cuda.synchronize()
+    assert kvr.kvr_sketch_device_status(sk) == 0
+    q_inst = qm.float().reshape(B, H, G, Qn, 128).reshape(n_inst, G, Qn, 128).numpy()
+    want = orc.decode_mq(q_inst, inst_major(Kr2), inst_major(Vr2), ret2.reshape(n_inst, -1).cpu().numpy(), cells_o,
+                         N0 + Qn, seeds, causal=causal)
+    got = out.reshape(B, H, G, Qn, 128).reshape(n_inst, G, Qn, 128).cpu().numpy()
+    assert np.isfinite(got).all()
+    assert np.abs(got - want).max() <= TOL, np.abs(got - want).max()
+    if Qn == 1:
+        single = kvr.kvr_decode_attention(sk, 0, qm[:, :, 0].contiguous().to(dev), Kr2, Vr2, ret2)
+        assert (single - out[:, :, 0]).abs().max().item() <= TOL
+    again = kvr.kvr_decode_attention_mq(sk, 0, qm.to(dev), Kr2, Vr2, ret2, causal=causal)      # bit-reproducible
+    assert torch.equal(out, again)
+    kvr.kvr_sketch_destroy(sk)
+
+
+def test_multi_query_decode_needs_a_class_grid():
+    """A handle with 8 query heads per kv head has no class grid: the multi-query call says so."""
+    seeds = synth.hash_seeds(3400)
+    K, V, Q, _ = make_case(3401, 1, 1, 8, 300, 4, F16, 1)
+    sk = kvr.kvr_sketch_create(b=5, batch=1, n_layers=1, n_kv_heads=1, n_q_heads=8, max_context=300, kv_dtype=F16,
+                               hash_seeds=seeds)
+    Kr, Vr, ret = kvr.kvr_compress(sk, 0, K[0].cuda(), V[0].cuda(), Q[0].cuda(), 30, 0)
+    qm = torch.randn((1, 8, 2, 128)).to(F16).cuda()
+    with pytest.raises(kvr.KvrError) as e:
+        kvr.kvr_decode_attention_mq(sk, 0, qm, Kr, Vr, ret, causal=False)
+    assert e.value.status == 2
+    kvr.kvr_sketch_destroy(sk)
+
+
 def test_per_layer_budgets_in_one_handle():
     """Budgets that differ from layer to layer (kvr_layer_budgets from per-layer weights): every layer
     of one handle is compressed with its own budget and decoded; selection, cells and outputs against
