@@ -568,6 +568,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="kvr", choices=["kvr", "reference"])
+    ap.add_argument("--all-workloads", action="store_true",
+                    help="one JSON line per benchmark workload (the budget x width sweep of 8k_qwen3_8b_batch8 included); "
+                         "no end-to-end and no CPU-baseline leg")
     ap.add_argument("--stream", type=int, default=0, help="time T generation steps with Algorithm 3 (kvr_append) instead")
     ap.add_argument("--queries", type=int, default=0, help="time decode attention with this many queries per head per call instead")
     ap.add_argument("--no-e2e", action="store_true")
@@ -587,6 +590,25 @@ def main():
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu dram bytes per decode launch to report in roofline.traffic (from profiles/)")
     args = ap.parse_args()
+    if args.all_workloads:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback of the hot path)")
+        rank, world, local = kdist.init_from_env()
+        args.no_e2e = args.no_cpu_baseline = True
+        args.warmup = max(args.warmup, 3)
+        points = [(n, 0.0, 0.0) for n in ("2k_single_layer", "2k_llama3_8b", "32k_llama3_8b", "32k_llama3_8b_batch16")]
+        points += [("8k_qwen3_8b_batch8", r, m) for r in (0.05, 0.10, 0.25, 0.50) for m in (0.5, 1.0, 2.0)]
+        for name, ratio, mult in points:
+            w = synth.WORKLOADS[name]
+            if ratio:
+                w = dataclasses.replace(w, budget_ratio=ratio, width_mult=mult, name=f"{name}[budget={ratio},width={mult}]")
+            result, inputs = run_gpu(args, w, rank, world, local)
+            del inputs
+            torch.cuda.empty_cache()
+            if rank == 0:
+                print(json.dumps(result), flush=True)
+        kdist.finalize()
+        return
     w = synth.WORKLOADS[args.workload]
     if args.layers or args.decode_steps:
         w = dataclasses.replace(w, n_layers=args.layers or w.n_layers, decode_steps=args.decode_steps or w.decode_steps,
