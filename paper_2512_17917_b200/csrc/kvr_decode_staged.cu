@@ -296,16 +296,26 @@ decode_staged_kernel(const StagedParams p) {
         bulk_g2s(smem_s + L.stage, clist + (s_begin - lshift), bytes, bar_list);
     }
     // The rows are read twice (keys, later values), microseconds apart: ask for all of them now, so
-    // that both reads find them in the L2 cache instead of waiting for HBM one batch at a time.
+    // that both reads find them in the L2 cache instead of waiting for HBM one batch at a time.  A
+    // request occupies its warp until the copy engine has taken it (about a microsecond per 8 KB
+    // when megabytes are asked for), so a CTA with many rows leaves all of them to its last warp,
+    // keys first, while the other warps start on the rows that have arrived.
     {
         constexpr int PF = 8192;                            // bytes per prefetch request (32 rows)
         const char* k8 = reinterpret_cast<const char*>(p.Kr + ((size_t)u * p.R + r_begin) * 32);
         const char* v8 = reinterpret_cast<const char*>(p.Vr + ((size_t)u * p.R + r_begin) * 32);
         const int bytes = (r_end - r_begin) * 256;
-        for (int o = (warp + lane * NW) * PF; o < bytes; o += NT * PF) {     // (dealt to the warps like the cell copies)
-            const uint32_t n = (uint32_t)min(PF, bytes - o);
-            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(k8 + o), "r"(n) : "memory");
-            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(v8 + o), "r"(n) : "memory");
+        if (bytes <= NW * PF) {
+            for (int o = (warp + lane * NW) * PF; o < bytes; o += NT * PF) {     // (dealt to the warps like the cell copies)
+                const uint32_t n = (uint32_t)min(PF, bytes - o);
+                asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(k8 + o), "r"(n) : "memory");
+                asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(v8 + o), "r"(n) : "memory");
+            }
+        } else if (warp == NW - 1) {
+            for (int o = lane * PF; o < bytes; o += 32 * PF)
+                asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(k8 + o), "r"((uint32_t)min(PF, bytes - o)) : "memory");
+            for (int o = lane * PF; o < bytes; o += 32 * PF)
+                asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(v8 + o), "r"((uint32_t)min(PF, bytes - o)) : "memory");
         }
     }
     // stretches: the tokens are taken lcap entries and rcap rows at a time (normally all at once)
