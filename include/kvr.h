@@ -78,6 +78,9 @@ typedef struct {
     int32_t index_mix;   /* 1: token indices are scrambled by a fixed 32-bit bijection before
                             hashing (default); 0: raw indices (test mode: seeds A=1,C=0 give
                             h(J) = J mod b, injective once b >= N)                               */
+    int32_t seeds_per_head; /* 0: one set of hash seeds for all head-instances; 1: one set per kv
+                            head (hash_seeds is then [n_kv_heads][r][4]): tokens collide in
+                            different cells in different heads                                  */
 } kvr_sketch_desc_t;
 
 typedef struct kvr_sketch kvr_sketch_t; /* opaque; library-owned host + device memory */
@@ -88,7 +91,9 @@ typedef struct kvr_sketch kvr_sketch_t; /* opaque; library-owned host + device m
  *     h_i(J) = ((A_i m(J) + C_i) mod p) mod b,   g_i(J) = +1 / -1 for (A'_i m(J) + C'_i) mod p
  *     even / odd,   p = 2^31 - 1,
  * with hash_seeds[i] = {A_i, C_i, A'_i, C'_i} (host, r x 4 uint32, each < p) shared by all
- * head-instances, and m the index scrambler selected by desc->index_mix.
+ * head-instances, or one such set per kv head (desc->seeds_per_head = 1: n_kv_heads x r x 4; the
+ * head-instances of a kv head share its set across batch and layers), and m the index scrambler
+ * selected by desc->index_mix.
  * Errors: INVALID_ARG (NULL, seed >= p, sizes < 1), UNSUPPORTED, ALLOC, CUDA.  *out is NULL on error. */
 kvr_status_t kvr_sketch_create(kvr_sketch_t** out, const kvr_sketch_desc_t* desc,
                                const uint32_t* hash_seeds, void* cuda_stream);

@@ -48,7 +48,7 @@ class KvrError(RuntimeError):
 class SketchDesc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "r", "b", "head_dim", "n_kv_heads", "n_q_heads", "batch", "n_layers", "max_context",
-        "kv_dtype", "index_mix")]
+        "kv_dtype", "index_mix", "seeds_per_head")]
 
 
 _lib = None
@@ -163,12 +163,13 @@ class Sketch:
 def kvr_sketch_create(*, b: int, batch: int, n_layers: int, n_kv_heads: int, n_q_heads: int,
                       max_context: int, kv_dtype: torch.dtype, hash_seeds, r: int = 3, head_dim: int = 128,
                       index_mix: bool = True, device="cuda", stream=None) -> Sketch:
-    """kvr_sketch_create: hash_seeds is an [r, 4] array of uint32 (A, C, A', C' per row)."""
+    """kvr_sketch_create: hash_seeds is an [r, 4] array of uint32 (A, C, A', C' per row), or
+    [n_kv_heads, r, 4] for one set of seeds per kv head."""
     seeds = np.ascontiguousarray(hash_seeds, dtype=np.uint32)
-    if seeds.shape != (r, 4):
-        raise ValueError("hash_seeds must have shape [r, 4]")
+    if seeds.shape not in ((r, 4), (n_kv_heads, r, 4)):
+        raise ValueError("hash_seeds must have shape [r, 4] or [n_kv_heads, r, 4]")
     desc = SketchDesc(r, b, head_dim, n_kv_heads, n_q_heads, batch, n_layers, max_context,
-                      _dtype_code(kv_dtype), int(bool(index_mix)))
+                      _dtype_code(kv_dtype), int(bool(index_mix)), int(seeds.ndim == 3))
     dev = torch.device(device)
     out = ctypes.c_void_p(0)
     with torch.cuda.device(dev):

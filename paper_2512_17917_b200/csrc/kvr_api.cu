@@ -195,7 +195,9 @@ kvr_status_t kvr_sketch_create(kvr_sketch_t** out, const kvr_sketch_desc_t* desc
     if (G != 1 && G != 2 && G != 4 && G != 8) return KVR_ERR_UNSUPPORTED;
     const long long n_inst = (long long)d.batch * d.n_layers * d.n_kv_heads;
     if (n_inst > 65535) return KVR_ERR_UNSUPPORTED;
-    for (int i = 0; i < KVR_R * 4; ++i)
+    if (d.seeds_per_head != 0 && d.seeds_per_head != 1) return KVR_ERR_INVALID_ARG;
+    const int n_tbl = d.seeds_per_head ? d.n_kv_heads : 1;
+    for (int i = 0; i < n_tbl * KVR_R * 4; ++i)
         if (hash_seeds[i] >= KVR_HASH_P) return KVR_ERR_INVALID_ARG;
 
     kvr_sketch* sk = new (std::nothrow) kvr_sketch();
@@ -204,7 +206,8 @@ kvr_status_t kvr_sketch_create(kvr_sketch_t** out, const kvr_sketch_desc_t* desc
     sk->G = G;
     sk->BH = d.batch * d.n_kv_heads;
     sk->n_inst = (int)n_inst;
-    memcpy(sk->seeds, hash_seeds, sizeof(sk->seeds));
+    sk->n_tbl = n_tbl;
+    sk->seeds.assign(hash_seeds, hash_seeds + (size_t)n_tbl * KVR_R * 4);
     sk->layer_N.assign(d.n_layers, -1);
     sk->layer_R.assign(d.n_layers, -1);
     if (cudaGetDevice(&sk->device) != cudaSuccess) { delete sk; return KVR_ERR_CUDA; }
@@ -236,11 +239,11 @@ kvr_status_t kvr_sketch_create(kvr_sketch_t** out, const kvr_sketch_desc_t* desc
     const size_t mc = (size_t)d.max_context, ni = (size_t)n_inst;
     kvr_status_t rc = KVR_OK;
     auto A = [&](auto** p, size_t bytes) { if (rc == KVR_OK) rc = dev_alloc(sk, p, bytes); };
-    A(&sk->tok_h, sizeof(int32_t) * KVR_R * mc);
-    A(&sk->tok_g, sizeof(int8_t) * KVR_R * mc);
-    A(&sk->tok_pack, sizeof(uint32_t) * mc);
-    A(&sk->full_off, sizeof(int32_t) * KVR_R * (d.b + 1));
-    A(&sk->full_list, sizeof(int32_t) * KVR_R * mc);
+    A(&sk->tok_h, sizeof(int32_t) * n_tbl * KVR_R * mc);
+    A(&sk->tok_g, sizeof(int8_t) * n_tbl * KVR_R * mc);
+    A(&sk->tok_pack, sizeof(uint32_t) * n_tbl * mc);
+    A(&sk->full_off, sizeof(int32_t) * n_tbl * KVR_R * (d.b + 1));
+    A(&sk->full_list, sizeof(int32_t) * n_tbl * KVR_R * mc);
     const size_t cell_bytes = sizeof(float) * ni * 2 * KVR_R * d.b * KVR_D;
     A(&sk->cells, cell_bytes);
     A(&sk->scores, sizeof(float) * ni * mc);

@@ -41,10 +41,11 @@ struct kvr_sketch {
     int n_inst;      // BH * n_layers
     int device;
     int n_sm;
-    uint32_t seeds[KVR_R][4];
+    int n_tbl;       // sets of hash tables: 1 (seeds shared by all heads) or n_kv_heads (seeds per kv head)
+    std::vector<uint32_t> seeds;   // [n_tbl][r][4]
 
     // ---- per-handle hash tables over token indices 0 .. max_context-1 (device) ----
-    int32_t* tok_h;      // [r][max_context]   cell of token J in row i
+    int32_t* tok_h;      // [n_tbl][r][max_context]   cell of token J in row i
     int8_t* tok_g;       // [r][max_context]   +1 / -1
     uint32_t* tok_pack;  // [max_context]      packed rows 1,2 + signs (see above)
     int32_t* full_off;   // [r][b+1]           CSR offsets: tokens of each cell, ascending

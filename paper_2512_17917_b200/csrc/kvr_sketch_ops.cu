@@ -19,7 +19,7 @@ __global__ void __launch_bounds__(INS_THREADS)
 insert_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ full_list,
               const int8_t* __restrict__ tok_g, const uint32_t* __restrict__ bitmap_all, int bitmap_words,
               const uint2* __restrict__ K, const uint2* __restrict__ V, int N, int max_ctx, int b,
-              int inst0, float* __restrict__ cells_all) {
+              int inst0, int n_tbl, float* __restrict__ cells_all) {
     __shared__ uint32_t s_tok[INS_THREADS];
     __shared__ int s_wcnt[INS_THREADS / 32];
     __shared__ float4 s_part[2][KVR_D / 4];      // sums of the odd tokens: [keys | values][4 channels]
@@ -28,8 +28,10 @@ insert_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int kv = warp & 1, par = warp >> 1;
     const uint32_t* bitmap = bitmap_all + (size_t)inst * bitmap_words;
-    const int32_t* list = full_list + (size_t)i * max_ctx;
-    const int8_t* g = tok_g + (size_t)i * max_ctx;
+    const int tb = n_tbl > 1 ? inst % n_tbl : 0;              // hash tables of this kv head (seeds per head) or the shared ones
+    full_off += (size_t)tb * KVR_R * (b + 1);
+    const int32_t* list = full_list + ((size_t)tb * KVR_R + i) * max_ctx;
+    const int8_t* g = tok_g + ((size_t)tb * KVR_R + i) * max_ctx;
     const uint2* src = (kv ? V : K) + (size_t)u * N * (KVR_D / 4) + lane;     // 4 channels (8 bytes) per lane
     const int p0 = full_off[i * (b + 1) + c], p1 = full_off[i * (b + 1) + c + 1];
 
@@ -108,9 +110,12 @@ insert_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ 
 // One warp per compressed token, 4 channels per lane.
 __global__ void reconstruct_kernel(const float* __restrict__ cells_all, const int32_t* __restrict__ cmp_all,
                                    const int32_t* __restrict__ tok_h, const int8_t* __restrict__ tok_g,
-                                   int max_ctx, int b, int a, int inst0, int mean, float* __restrict__ Kt,
+                                   int max_ctx, int b, int a, int inst0, int n_tbl, int mean, float* __restrict__ Kt,
                                    float* __restrict__ Vt) {
     const int u = blockIdx.y, inst = inst0 + u;
+    const int tb = n_tbl > 1 ? inst % n_tbl : 0;
+    tok_h += (size_t)tb * KVR_R * max_ctx;
+    tok_g += (size_t)tb * KVR_R * max_ctx;
     const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (t >= a) return;
@@ -143,12 +148,12 @@ cudaError_t kvr_launch_insert(kvr_sketch* sk, int inst0, int n_inst, int N, cons
     if (sk->d.kv_dtype == KVR_F16)
         insert_kernel<__half><<<g, INS_THREADS, 0, st>>>(sk->full_off, sk->full_list, sk->tok_g, sk->bitmap,
                                                          sk->bitmap_words, (const uint2*)K, (const uint2*)V,
-                                                         N, sk->d.max_context, sk->d.b, inst0, sk->cells);
+                                                         N, sk->d.max_context, sk->d.b, inst0, sk->n_tbl, sk->cells);
     else
         insert_kernel<__nv_bfloat16><<<g, INS_THREADS, 0, st>>>(sk->full_off, sk->full_list, sk->tok_g, sk->bitmap,
                                                                 sk->bitmap_words, (const uint2*)K,
                                                                 (const uint2*)V, N, sk->d.max_context,
-                                                                sk->d.b, inst0, sk->cells);
+                                                                sk->d.b, inst0, sk->n_tbl, sk->cells);
     sk->launches += 1;
     return cudaGetLastError();
 }
@@ -158,7 +163,7 @@ cudaError_t kvr_launch_reconstruct(const kvr_sketch* sk, int inst0, int n_inst, 
     if (a <= 0 || n_inst <= 0) return cudaSuccess;
     dim3 g((a + 7) / 8, n_inst);
     reconstruct_kernel<<<g, 256, 0, st>>>(sk->cells, sk->cmp_idx, sk->tok_h, sk->tok_g, sk->d.max_context,
-                                          sk->d.b, a, inst0, sk->combine, Kt, Vt);
+                                          sk->d.b, a, inst0, sk->n_tbl, sk->combine, Kt, Vt);
     const_cast<kvr_sketch*>(sk)->launches += 1;
     return cudaGetLastError();
 }

@@ -55,8 +55,9 @@ template <typename T, int G>
 __global__ void __launch_bounds__(256)
 vague_mass_kernel(const uint2* __restrict__ q, const float* __restrict__ cells_all, const int32_t* __restrict__ cmp_all,
                   const int32_t* __restrict__ tok_h, const float* __restrict__ ml_all, int max_ctx, int b, int a,
-                  int inst0, int mean, float scale_log2e, float* __restrict__ scores_all) {
+                  int inst0, int n_tbl, int mean, float scale_log2e, float* __restrict__ scores_all) {
     const int u = blockIdx.y, inst = inst0 + u, lane = threadIdx.x & 31;
+    tok_h += (size_t)(n_tbl > 1 ? inst % n_tbl : 0) * KVR_R * max_ctx;
     const int t = blockIdx.x * 8 + (threadIdx.x >> 5);
     if (t >= a) return;                                           // (whole warp)
     const int J = cmp_all[(size_t)inst * max_ctx + t];
@@ -115,10 +116,12 @@ swap_kernel(T* __restrict__ Kr_all, T* __restrict__ Vr_all, int32_t* __restrict_
             int rows, int n_recent, float rate, int max_swaps, float* __restrict__ scores_all,
             int32_t* __restrict__ cmp_all, int a, uint32_t* __restrict__ bitmap_all, int bitmap_words,
             float* __restrict__ cells_all, const int32_t* __restrict__ tok_h, const int8_t* __restrict__ tok_g,
-            int max_ctx, int b, int inst0, int mean, int32_t* __restrict__ n_swapped) {
+            int max_ctx, int b, int inst0, int n_tbl, int mean, int32_t* __restrict__ n_swapped) {
     __shared__ unsigned long long s_w[32];
     __shared__ int s_row, s_pos;
     const int u = blockIdx.x, inst = inst0 + u, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    tok_h += (size_t)(n_tbl > 1 ? inst % n_tbl : 0) * KVR_R * max_ctx;
+    tok_g += (size_t)(n_tbl > 1 ? inst % n_tbl : 0) * KVR_R * max_ctx;
     T* Kr = Kr_all + (size_t)u * rows * KVR_D;
     T* Vr = Vr_all + (size_t)u * rows * KVR_D;
     int32_t* ret = ret_all + (size_t)u * rows;
@@ -232,8 +235,10 @@ __global__ void __launch_bounds__(128)
 insert_rows_kernel(const int32_t* __restrict__ tok_h, const int8_t* __restrict__ tok_g,
                    const int32_t* __restrict__ ev_tok, const int32_t* __restrict__ evict_pos,
                    const uint32_t* __restrict__ Kr, const uint32_t* __restrict__ Vr, int rows, int n_ev, int max_ctx,
-                   int b, int inst0, float* __restrict__ cells_all) {
+                   int b, int inst0, int n_tbl, float* __restrict__ cells_all) {
     const int c = blockIdx.x, i = blockIdx.y, u = blockIdx.z, inst = inst0 + u;
+    tok_h += (size_t)(n_tbl > 1 ? inst % n_tbl : 0) * KVR_R * max_ctx;
+    tok_g += (size_t)(n_tbl > 1 ? inst % n_tbl : 0) * KVR_R * max_ctx;
     const int tid = threadIdx.x, half = tid >> 6, c2 = tid & 63;
     const int32_t* h = tok_h + (size_t)i * max_ctx;
     const int8_t* g = tok_g + (size_t)i * max_ctx;
@@ -350,7 +355,7 @@ cudaError_t kvr_launch_vague_mass(kvr_sketch* sk, int inst0, int n_inst, int a, 
     const dim3 grid((a + 7) / 8, n_inst);
     const float sl = scale * 1.4426950408889634f;
     const bool f16 = sk->d.kv_dtype == KVR_F16;
-#define KVR_VM(TT, GG) vague_mass_kernel<TT, GG><<<grid, 256, 0, st>>>((const uint2*)q, sk->cells, sk->cmp_idx, sk->tok_h, sk->ml, sk->d.max_context, sk->d.b, a, inst0, sk->combine, sl, sk->scores)
+#define KVR_VM(TT, GG) vague_mass_kernel<TT, GG><<<grid, 256, 0, st>>>((const uint2*)q, sk->cells, sk->cmp_idx, sk->tok_h, sk->ml, sk->d.max_context, sk->d.b, a, inst0, sk->n_tbl, sk->combine, sl, sk->scores)
     switch (sk->G) {
         case 1: if (f16) KVR_VM(__half, 1); else KVR_VM(__nv_bfloat16, 1); break;
         case 2: if (f16) KVR_VM(__half, 2); else KVR_VM(__nv_bfloat16, 2); break;
@@ -371,12 +376,12 @@ cudaError_t kvr_launch_swap(kvr_sketch* sk, int inst0, int n_inst, int N, int a,
     if (sk->d.kv_dtype == KVR_F16)
         swap_kernel<__half><<<n_inst, 1024, 0, st>>>((__half*)Kr, (__half*)Vr, ret_idx, row_scores, rows, n_recent, rate,
                                                      max_swaps, sk->scores, sk->cmp_idx, a, sk->bitmap, sk->bitmap_words,
-                                                     sk->cells, sk->tok_h, sk->tok_g, mc, sk->d.b, inst0, sk->combine, n_swapped);
+                                                     sk->cells, sk->tok_h, sk->tok_g, mc, sk->d.b, inst0, sk->n_tbl, sk->combine, n_swapped);
     else
         swap_kernel<__nv_bfloat16><<<n_inst, 1024, 0, st>>>((__nv_bfloat16*)Kr, (__nv_bfloat16*)Vr, ret_idx, row_scores,
                                                             rows, n_recent, rate, max_swaps, sk->scores, sk->cmp_idx, a,
                                                             sk->bitmap, sk->bitmap_words, sk->cells, sk->tok_h,
-                                                            sk->tok_g, mc, sk->d.b, inst0, sk->combine, n_swapped);
+                                                            sk->tok_g, mc, sk->d.b, inst0, sk->n_tbl, sk->combine, n_swapped);
     cmp_from_bitmap_kernel<<<n_inst, 1024, 0, st>>>(sk->bitmap, sk->bitmap_words, N, mc, inst0, sk->cmp_idx);
     sk->launches += 2;
     cudaError_t e = cudaGetLastError();
@@ -413,11 +418,11 @@ cudaError_t kvr_launch_demote(kvr_sketch* sk, int inst0, int n_inst, int rows, i
         const dim3 g(b, KVR_R, n_inst);
         if (sk->d.kv_dtype == KVR_F16)
             insert_rows_kernel<__half><<<g, 128, 0, st>>>(sk->tok_h, sk->tok_g, ev_tok, evict_pos, (const uint32_t*)Kr,
-                                                          (const uint32_t*)Vr, rows, n_ev, mc, b, inst0, sk->cells);
+                                                          (const uint32_t*)Vr, rows, n_ev, mc, b, inst0, sk->n_tbl, sk->cells);
         else
             insert_rows_kernel<__nv_bfloat16><<<g, 128, 0, st>>>(sk->tok_h, sk->tok_g, ev_tok, evict_pos,
                                                                  (const uint32_t*)Kr, (const uint32_t*)Vr, rows, n_ev,
-                                                                 mc, b, inst0, sk->cells);
+                                                                 mc, b, inst0, sk->n_tbl, sk->cells);
     }
     cmp_from_bitmap_kernel<<<n_inst, 1024, 0, st>>>(sk->bitmap, sk->bitmap_words, N_new, mc, inst0, sk->cmp_idx);
     sk->launches += 2 + (n_ev > 0 ? 1 : 0);

@@ -123,7 +123,7 @@ constexpr int LST_CL = 8, LST_THREADS = 1024;
 __global__ void __cluster_dims__(LST_CL, 1, 1) __launch_bounds__(LST_THREADS, 1)
 lists_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ full_list,
              const uint32_t* __restrict__ tok_pack, const uint32_t* __restrict__ bitmap_all, int bitmap_words,
-             int b, int N, int max_ctx, int inst0, int C, int logC, int n1, uint32_t* __restrict__ dlist_all,
+             int b, int N, int max_ctx, int inst0, int n_tbl, int C, int logC, int n1, uint32_t* __restrict__ dlist_all,
              int32_t* __restrict__ doff_all, uint2* __restrict__ clist_all, int32_t* __restrict__ coff_all) {
     extern __shared__ int32_t s_cnt[];        // [cells of this CTA][1 + C * C]: kept tokens, then per class
     __shared__ int32_t s_tot[65];             // column sums over this CTA's cells
@@ -134,6 +134,12 @@ lists_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ f
     cg::cluster_group cluster = cg::this_cluster();
     const int crank = (int)cluster.block_rank();
     const int inst = inst0 + blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    {
+        const int tb = n_tbl > 1 ? inst % n_tbl : 0;            // hash tables of this kv head, or the shared ones
+        full_off += (size_t)tb * KVR_R * (b + 1);
+        full_list += (size_t)tb * KVR_R * max_ctx;
+        tok_pack += (size_t)tb * max_ctx;
+    }
     const int n_cls = C * C, n_col = 1 + n_cls;
     const int bc = (b + LST_CL - 1) / LST_CL;
     const int c_lo = min(crank * bc, b), c_hi = min(c_lo + bc, b), n_c = c_hi - c_lo;
@@ -286,12 +292,15 @@ lists_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ f
 }
 
 __global__ void assignment_kernel(const int32_t* __restrict__ cmp_all, const int32_t* __restrict__ tok_h,
-                                  const int8_t* __restrict__ tok_g, int max_ctx, int a, int inst0,
+                                  const int8_t* __restrict__ tok_g, int max_ctx, int a, int inst0, int n_tbl,
                                   int32_t* __restrict__ cmp_out, int32_t* __restrict__ bucket,
                                   int8_t* __restrict__ sign) {
     int t = blockIdx.x * blockDim.x + threadIdx.x;
     int u = blockIdx.y;
     if (t >= a) return;
+    const int tb = n_tbl > 1 ? (inst0 + u) % n_tbl : 0;
+    tok_h += (size_t)tb * KVR_R * max_ctx;
+    tok_g += (size_t)tb * KVR_R * max_ctx;
     int J = cmp_all[(size_t)(inst0 + u) * max_ctx + t];
     if (cmp_out) cmp_out[(size_t)u * a + t] = J;
 #pragma unroll
@@ -305,19 +314,25 @@ __global__ void assignment_kernel(const int32_t* __restrict__ cmp_all, const int
 
 cudaError_t kvr_launch_hash_tables(kvr_sketch* sk, cudaStream_t st) {
     const int b = sk->d.b, mc = sk->d.max_context;
-    SeedPack sp;
-    for (int i = 0; i < KVR_R; ++i)
-        for (int k = 0; k < 4; ++k) sp.s[i][k] = sk->seeds[i][k];
     int32_t* cnt = nullptr;
     cudaError_t e = cudaMalloc(&cnt, sizeof(int32_t) * KVR_R * b);
     if (e != cudaSuccess) return e;
-    hash_table_kernel<<<(mc + 255) / 256, 256, 0, st>>>(sp, sk->d.index_mix, b, mc, sk->tok_h, sk->tok_g,
-                                                        sk->tok_pack);
-    dim3 g((b + 127) / 128, KVR_R);
-    csr_count_kernel<<<g, 128, 0, st>>>(sk->tok_h, b, mc, cnt);
-    csr_scan_kernel<<<KVR_R, 1024, 0, st>>>(cnt, b, sk->full_off);
-    csr_fill_kernel<<<g, 128, 0, st>>>(sk->tok_h, sk->full_off, b, mc, sk->full_list);
-    sk->launches += 4;
+    for (int t = 0; t < sk->n_tbl; ++t) {                       // one set of tables per kv head, or one for all
+        SeedPack sp;
+        for (int i = 0; i < KVR_R; ++i)
+            for (int k = 0; k < 4; ++k) sp.s[i][k] = sk->seeds[((size_t)t * KVR_R + i) * 4 + k];
+        int32_t* tok_h = sk->tok_h + (size_t)t * KVR_R * mc;
+        int8_t* tok_g = sk->tok_g + (size_t)t * KVR_R * mc;
+        int32_t* full_off = sk->full_off + (size_t)t * KVR_R * (b + 1);
+        int32_t* full_list = sk->full_list + (size_t)t * KVR_R * mc;
+        hash_table_kernel<<<(mc + 255) / 256, 256, 0, st>>>(sp, sk->d.index_mix, b, mc, tok_h, tok_g,
+                                                            sk->tok_pack + (size_t)t * mc);
+        dim3 g((b + 127) / 128, KVR_R);
+        csr_count_kernel<<<g, 128, 0, st>>>(tok_h, b, mc, cnt);
+        csr_scan_kernel<<<KVR_R, 1024, 0, st>>>(cnt, b, full_off);
+        csr_fill_kernel<<<g, 128, 0, st>>>(tok_h, full_off, b, mc, full_list);
+        sk->launches += 4;
+    }
     e = cudaStreamSynchronize(st);
     cudaFree(cnt);
     if (e != cudaSuccess) return e;
@@ -330,7 +345,7 @@ cudaError_t kvr_launch_lists(kvr_sketch* sk, int inst0, int n_inst, int N, cudaS
     const int bc = (b + LST_CL - 1) / LST_CL;
     const size_t smem = sizeof(int32_t) * (size_t)bc * (1 + C * C);
     lists_kernel<<<dim3(LST_CL, n_inst), LST_THREADS, smem, st>>>(sk->full_off, sk->full_list, sk->tok_pack, sk->bitmap,
-                                                                  sk->bitmap_words, b, N, sk->d.max_context, inst0, C,
+                                                                  sk->bitmap_words, b, N, sk->d.max_context, inst0, sk->n_tbl, C,
                                                                   sk->logC, sk->n1, sk->dlist, sk->doff, sk->clist,
                                                                   sk->coff);
     sk->launches += 1;
@@ -341,7 +356,7 @@ cudaError_t kvr_launch_assignment(const kvr_sketch* sk, int inst0, int n_inst, i
                                   int32_t* bucket, int8_t* sign, cudaStream_t st) {
     if (a <= 0 || n_inst <= 0) return cudaSuccess;
     dim3 g((a + 255) / 256, n_inst);
-    assignment_kernel<<<g, 256, 0, st>>>(sk->cmp_idx, sk->tok_h, sk->tok_g, sk->d.max_context, a, inst0,
+    assignment_kernel<<<g, 256, 0, st>>>(sk->cmp_idx, sk->tok_h, sk->tok_g, sk->d.max_context, a, inst0, sk->n_tbl,
                                          cmp_idx, bucket, sign);
     const_cast<kvr_sketch*>(sk)->launches += 1;
     return cudaGetLastError();

@@ -35,7 +35,7 @@ def test_status_strings():
 
 def _create(**over):
     kw = dict(r=3, b=8, head_dim=128, n_kv_heads=2, n_q_heads=8, batch=1, n_layers=1, max_context=64,
-              kv_dtype=0, index_mix=1)
+              kv_dtype=0, index_mix=1, seeds_per_head=0)
     kw.update(over)
     desc = binding.SketchDesc(*[kw[n] for n, _ in binding.SketchDesc._fields_])
     seeds = over.get("_seeds", synth.hash_seeds(1))
@@ -49,7 +49,7 @@ def _create(**over):
 
 @pytest.mark.parametrize("over,status", [
     (dict(b=0), 1), (dict(batch=0), 1), (dict(max_context=0), 1), (dict(kv_dtype=7), 1),
-    (dict(n_q_heads=7), 1), (dict(index_mix=2), 1),
+    (dict(n_q_heads=7), 1), (dict(index_mix=2), 1), (dict(seeds_per_head=2), 1),
     (dict(r=5), 2), (dict(head_dim=64), 2), (dict(b=8193), 2), (dict(n_q_heads=6), 2),
     (dict(batch=4096, n_layers=64), 2),
 ])

@@ -493,6 +493,77 @@ def test_multi_query_decode_needs_a_class_grid():
     kvr.kvr_sketch_destroy(sk)
 
 
+@pytest.mark.parametrize("which", ["staged", "split"])
+def test_hash_seeds_per_kv_head(which):
+    """One set of hash seeds per kv head (the head-instances of a kv head share it across batch and
+    layers): bucket and sign assignment, cells, reconstruction, decode, the attention mass of vague
+    tokens, an overflow step and several queries per head, each head-instance against the oracle run
+    with its own head's seeds; the heads really hash differently."""
+    B, H, Hq, L, N, W, R, b = 2, 2, 8, 2, 1100, 8, 120, 13
+    G = Hq // H
+    n_inst = L * B * H
+    seeds = np.stack([synth.hash_seeds(7100), synth.hash_seeds(7200)])           # [H, r, 4]
+    K, V, Q, q = make_case(7001, B, H, Hq, N + 6, W, F16, L)
+    dev = "cuda"
+    sk = kvr.kvr_sketch_create(b=b, batch=B, n_layers=L, n_kv_heads=H, n_q_heads=Hq, max_context=N + 6, kv_dtype=F16,
+                               hash_seeds=seeds)
+    kvr.kvr_sketch_set_decode_kernel(sk, kvr.KVR_DECODE_SPLIT if which == "split" else kvr.KVR_DECODE_STAGED)
+    Kd, Vd = K[:, :, :, :N].contiguous().to(dev), V[:, :, :, :N].contiguous().to(dev)
+    Kr, Vr, ret = kvr.kvr_compress(sk, kvr.KVR_ALL_LAYERS, Kd, Vd, Q.to(dev), R, 5)
+    out = kvr.kvr_decode_attention(sk, kvr.KVR_ALL_LAYERS, q.to(dev), Kr, Vr, ret)
+    cmp_g, bk_g, sg_g = (x.cpu().numpy() for x in kvr.kvr_get_assignment(sk, kvr.KVR_ALL_LAYERS))
+    cells_g = kvr.kvr_get_cells(sk, kvr.KVR_ALL_LAYERS).reshape(n_inst, 2, 3, b, 128).cpu().numpy().transpose(0, 2, 3, 1, 4)
+    Kt_g, Vt_g = (x.reshape(n_inst, N - R, 128).cpu().numpy() for x in kvr.kvr_reconstruct(sk, kvr.KVR_ALL_LAYERS))
+    assert kvr.kvr_sketch_device_status(sk) == 0
+    Kc, Vc = inst_major(K)[:, :N], inst_major(V)[:, :N]
+    qc = dec_to_inst(q, H)
+    cmp_g, bk_g, sg_g = cmp_g.reshape(n_inst, -1), bk_g.reshape(n_inst, 3, -1), sg_g.reshape(n_inst, 3, -1)
+    ret_np, out_np = ret.reshape(n_inst, R).cpu().numpy(), out.reshape(n_inst, G, 128).cpu().numpy()
+    Kr_np, Vr_np = inst_major(Kr), inst_major(Vr)
+    cells_o = []
+    for u in range(n_inst):
+        sd = seeds[u % H]
+        bo, so = orc.bucket_sign(cmp_g[u], sd, b)
+        assert (bk_g[u] == bo).all() and (sg_g[u] == so).all()
+        co = orc.insert(Kc[u:u + 1], Vc[u:u + 1], cmp_g[u:u + 1], sd, b)
+        cells_o.append(co[0])
+        assert np.abs(cells_g[u] - co[0]).max() <= TOL
+        Kt_o, Vt_o = orc.query(co, cmp_g[u:u + 1], sd)
+        assert np.abs(Kt_g[u] - Kt_o[0]).max() <= TOL and np.abs(Vt_g[u] - Vt_o[0]).max() <= TOL
+        want = orc.decode(qc[u:u + 1], Kr_np[u:u + 1], Vr_np[u:u + 1], ret_np[u:u + 1], co, N, sd)
+        assert np.abs(out_np[u] - want[0]).max() <= TOL
+    u0, u1 = 0, 1                                                               # same batch element and layer, heads 0 and 1
+    both = np.intersect1d(cmp_g[u0], cmp_g[u1])
+    i0, i1 = np.searchsorted(cmp_g[u0], both), np.searchsorted(cmp_g[u1], both)
+    assert (bk_g[u0][:, i0] != bk_g[u1][:, i1]).mean() > 0.5                   # different hash functions per head
+    # ---- several queries per head (layer 1) and the streaming side (layer 0) use the same tables
+    if which == "staged":
+        gen = torch.Generator().manual_seed(7002)
+        qm = torch.randn((B, Hq, 3, 128), generator=gen).to(F16)
+        om = kvr.kvr_decode_attention_mq(sk, 1, qm.to(dev), Kr[1], Vr[1], ret[1], causal=False)
+        qmi = qm.float().reshape(B, H, G, 3, 128).reshape(B * H, G, 3, 128).numpy()
+        for k in range(B * H):
+            u = B * H + k
+            want = orc.decode_mq(qmi[k:k + 1], Kr_np[u:u + 1], Vr_np[u:u + 1], ret_np[u:u + 1], cells_o[u][None], N, seeds[u % H],
+                                 causal=False)
+            assert np.abs(om.reshape(B * H, G, 3, 128).cpu().numpy()[k] - want[0]).max() <= TOL
+    s0 = kvr.kvr_get_scores(sk, 0).reshape(B * H, -1)
+    acc = torch.gather(s0, 1, ret[0].reshape(B * H, -1).long()).reshape(B, H, R).contiguous()
+    Kn, Vn = K[0, :, :, N:N + 6].contiguous().to(dev), V[0, :, :, N:N + 6].contiguous().to(dev)
+    acc_np = acc.reshape(B * H, -1).cpu().numpy()
+    tok_np = s0.cpu().numpy()
+    Ko, Vo, ro, so, rec, n_sw = kvr.kvr_append(sk, 0, Kr[0], Vr[0], ret[0], acc, 5, Kn, Vn, 4, R - 10, 2, 1.1, 8)
+    cells_a = kvr.kvr_get_cells(sk, 0).reshape(B * H, 2, 3, b, 128).cpu().numpy().transpose(0, 2, 3, 1, 4)
+    for u in range(B * H):
+        tok_u = np.concatenate([tok_np[u], np.zeros(6, np.float32)])
+        got = orc.compress_stream(Kr_np[u], Vr_np[u], ret_np[u], acc_np[u], 5, tok_u, cells_o[u], inst_major(K[0])[u, N:N + 6],
+                                  inst_major(V[0])[u, N:N + 6], np.arange(N, N + 6, dtype=np.int32), 4, R - 10, 2, 1.1, 8,
+                                  seeds[u % H], round_rows=lambda x: torch.from_numpy(np.asarray(x, np.float64)).to(F16).double().numpy())
+        assert (ro.reshape(B * H, -1).cpu().numpy()[u] == got[2]).all() and got[4] == rec
+        assert np.abs(cells_a[u] - got[6]).max() <= TOL
+    kvr.kvr_sketch_destroy(sk)
+
+
 def test_per_layer_budgets_in_one_handle():
     """Budgets that differ from layer to layer (kvr_layer_budgets from per-layer weights): every layer
     of one handle is compressed with its own budget and decoded; selection, cells and outputs against
