@@ -50,7 +50,7 @@ extern "C" {
 typedef enum {
     KVR_OK = 0,
     KVR_ERR_INVALID_ARG = 1, /* NULL / misaligned pointer, value out of range */
-    KVR_ERR_UNSUPPORTED = 2, /* legal in the paper, not built here (r != 3, head_dim != 128, ...) */
+    KVR_ERR_UNSUPPORTED = 2, /* legal in the paper, not built here (r = 7, head_dim != 128, ...)   */
     KVR_ERR_SHAPE = 3,       /* sizes inconsistent with the handle (N > max_context, layer, ...) */
     KVR_ERR_ALLOC = 4,       /* device allocation failed */
     KVR_ERR_CUDA = 5,        /* a CUDA runtime call or launch failed */
@@ -66,7 +66,9 @@ typedef enum { KVR_F16 = 0, KVR_BF16 = 1 } kvr_dtype_t;
 /* Shape of the Vague sketch and of the model slice it serves (Vague Sketch section: r rows of
  * b cells, each cell a key vector and a value vector of head_dim elements, all zero initially). */
 typedef struct {
-    int32_t r;           /* rows ("buckets" in the paper); only 3, the paper's fixed value       */
+    int32_t r;           /* rows ("buckets" in the paper): 3 (the paper's fixed value; the fast
+                            kernels), or 1 / 5 (a general kernel; compress, decode and the
+                            inspection calls only)                                               */
     int32_t b;           /* cells per row, 1 .. KVR_MAX_B                                        */
     int32_t head_dim;    /* d_k; only 128                                                        */
     int32_t n_kv_heads;  /* H                                                                    */

@@ -134,7 +134,8 @@ kvr_status_t compress_impl(kvr_sketch* sk, const LayerRange& lr, const void* K, 
     KVR_CUDA(cudaStreamWaitEvent(sk->side, sk->ev_fork, 0));
     // The side stream has forked: whatever happens next, it is joined again before this call returns
     // (an unjoined fork would break a stream capture and let the next call race with the lists kernel).
-    cudaError_t e = kvr_launch_lists(sk, lr.inst0, lr.n_inst, N, sk->side);
+    // (the token lists feed the r = 3 decode kernels; other r walk the compressed-index list)
+    cudaError_t e = sk->d.r == KVR_R ? kvr_launch_lists(sk, lr.inst0, lr.n_inst, N, sk->side) : cudaSuccess;
     const cudaError_t e_rec = cudaEventRecord(sk->ev_join, sk->side);
     if (e == cudaSuccess) e = kvr_launch_gather(sk, lr.n_inst, N, R, K, V, ret_idx, Kr, Vr, st);
     if (e == cudaSuccess) e = kvr_launch_insert(sk, lr.inst0, lr.n_inst, N, K, V, st);
@@ -148,6 +149,16 @@ kvr_status_t compress_impl(kvr_sketch* sk, const LayerRange& lr, const void* K, 
 kvr_status_t decode_impl(kvr_sketch* sk, const LayerRange& lr, int N, int R, int rows, const void* q, const void* Kr,
                          const void* Vr, float scale, float* out, cudaStream_t st) {
     if (scale == 0.f) scale = (float)(1.0 / sqrt((double)sk->d.head_dim));
+    if (sk->d.r != KVR_R) {                        // r = 1 or 5: the general kernel
+        if (sk->decode_kernel == KVR_DECODE_STAGED) return KVR_ERR_UNSUPPORTED;
+        const int S = kvr_decode_pick_splits(sk, lr.n_inst, N, R);
+        kvr_status_t rc = ensure(sk, &sk->ws_decode, &sk->ws_decode_bytes, kvr_decode_ws_bytes(lr.n_inst, S, sk->G));
+        if (rc != KVR_OK) return rc;
+        sk->chain = false;
+        KVR_CUDA(kvr_launch_decode_generic(sk, lr.inst0, lr.n_inst, N, R, rows, q, Kr, Vr, scale, out, S, st));
+        sk->last_decode_kernel = KVR_DECODE_SPLIT;
+        return KVR_OK;
+    }
     KvrStagedPlan plan;
     if (sk->decode_kernel != KVR_DECODE_SPLIT &&
         kvr_decode_staged_plan(sk, lr.n_inst, N, R, rows, sk->decode_kernel == KVR_DECODE_STAGED, &plan)) {
@@ -191,13 +202,13 @@ kvr_status_t kvr_sketch_create(kvr_sketch_t** out, const kvr_sketch_desc_t* desc
     if (d.index_mix != 0 && d.index_mix != 1) return KVR_ERR_INVALID_ARG;
     if (d.n_q_heads % d.n_kv_heads != 0) return KVR_ERR_INVALID_ARG;
     const int G = d.n_q_heads / d.n_kv_heads;
-    if (d.r != KVR_R || d.head_dim != KVR_D || d.b > KVR_MAX_B) return KVR_ERR_UNSUPPORTED;
+    if ((d.r != 1 && d.r != 3 && d.r != 5) || d.head_dim != KVR_D || d.b > KVR_MAX_B) return KVR_ERR_UNSUPPORTED;
     if (G != 1 && G != 2 && G != 4 && G != 8) return KVR_ERR_UNSUPPORTED;
     const long long n_inst = (long long)d.batch * d.n_layers * d.n_kv_heads;
     if (n_inst > 65535) return KVR_ERR_UNSUPPORTED;
     if (d.seeds_per_head != 0 && d.seeds_per_head != 1) return KVR_ERR_INVALID_ARG;
     const int n_tbl = d.seeds_per_head ? d.n_kv_heads : 1;
-    for (int i = 0; i < n_tbl * KVR_R * 4; ++i)
+    for (int i = 0; i < n_tbl * d.r * 4; ++i)
         if (hash_seeds[i] >= KVR_HASH_P) return KVR_ERR_INVALID_ARG;
 
     kvr_sketch* sk = new (std::nothrow) kvr_sketch();
@@ -207,7 +218,7 @@ kvr_status_t kvr_sketch_create(kvr_sketch_t** out, const kvr_sketch_desc_t* desc
     sk->BH = d.batch * d.n_kv_heads;
     sk->n_inst = (int)n_inst;
     sk->n_tbl = n_tbl;
-    sk->seeds.assign(hash_seeds, hash_seeds + (size_t)n_tbl * KVR_R * 4);
+    sk->seeds.assign(hash_seeds, hash_seeds + (size_t)n_tbl * d.r * 4);
     sk->layer_N.assign(d.n_layers, -1);
     sk->layer_R.assign(d.n_layers, -1);
     if (cudaGetDevice(&sk->device) != cudaSuccess) { delete sk; return KVR_ERR_CUDA; }
@@ -215,7 +226,7 @@ kvr_status_t kvr_sketch_create(kvr_sketch_t** out, const kvr_sketch_desc_t* desc
     if (cudaGetDeviceProperties(&prop, sk->device) != cudaSuccess) { delete sk; return KVR_ERR_CUDA; }
     sk->n_sm = prop.multiProcessorCount;
     sk->bitmap_words = (d.max_context + 31) / 32;
-    sk->C = kvr_decode_staged_pick_C(d.b, G);
+    sk->C = d.r == KVR_R ? kvr_decode_staged_pick_C(d.b, G) : 0;
     sk->logC = 0;
     while ((1 << sk->logC) < sk->C) ++sk->logC;
     sk->n1 = sk->C > 0 ? (d.b + sk->C - 1) / sk->C : 0;
@@ -239,12 +250,12 @@ kvr_status_t kvr_sketch_create(kvr_sketch_t** out, const kvr_sketch_desc_t* desc
     const size_t mc = (size_t)d.max_context, ni = (size_t)n_inst;
     kvr_status_t rc = KVR_OK;
     auto A = [&](auto** p, size_t bytes) { if (rc == KVR_OK) rc = dev_alloc(sk, p, bytes); };
-    A(&sk->tok_h, sizeof(int32_t) * n_tbl * KVR_R * mc);
-    A(&sk->tok_g, sizeof(int8_t) * n_tbl * KVR_R * mc);
+    A(&sk->tok_h, sizeof(int32_t) * n_tbl * d.r * mc);
+    A(&sk->tok_g, sizeof(int8_t) * n_tbl * d.r * mc);
     A(&sk->tok_pack, sizeof(uint32_t) * n_tbl * mc);
-    A(&sk->full_off, sizeof(int32_t) * n_tbl * KVR_R * (d.b + 1));
-    A(&sk->full_list, sizeof(int32_t) * n_tbl * KVR_R * mc);
-    const size_t cell_bytes = sizeof(float) * ni * 2 * KVR_R * d.b * KVR_D;
+    A(&sk->full_off, sizeof(int32_t) * n_tbl * d.r * (d.b + 1));
+    A(&sk->full_list, sizeof(int32_t) * n_tbl * d.r * mc);
+    const size_t cell_bytes = sizeof(float) * ni * 2 * d.r * d.b * KVR_D;
     A(&sk->cells, cell_bytes);
     A(&sk->scores, sizeof(float) * ni * mc);
     A(&sk->cmp_idx, sizeof(int32_t) * ni * mc);
@@ -279,9 +290,9 @@ kvr_status_t kvr_sketch_reset(kvr_sketch_t* sk, int32_t layer, void* cuda_stream
     LayerRange lr;
     kvr_status_t rc = layer_range(sk, layer, &lr);
     if (rc != KVR_OK) return rc;
-    const size_t per = sizeof(float) * 2 * KVR_R * sk->d.b * KVR_D;
+    const size_t per = sizeof(float) * 2 * sk->d.r * sk->d.b * KVR_D;
     sk->chain = false;
-    KVR_CUDA(cudaMemsetAsync(sk->cells + (size_t)lr.inst0 * 2 * KVR_R * sk->d.b * KVR_D, 0, per * lr.n_inst,
+    KVR_CUDA(cudaMemsetAsync(sk->cells + (size_t)lr.inst0 * 2 * sk->d.r * sk->d.b * KVR_D, 0, per * lr.n_inst,
                              (cudaStream_t)cuda_stream));
     for (int l = lr.layer0; l < lr.layer0 + lr.n_layers; ++l) sk->layer_N[l] = sk->layer_R[l] = -1;
     return KVR_OK;
@@ -390,6 +401,7 @@ kvr_status_t kvr_accumulate_vague_scores(kvr_sketch_t* sk, int32_t layer, const 
                                          void* cuda_stream) {
     if (!sk || !q || !aligned16(q)) return KVR_ERR_INVALID_ARG;
     if (!(softmax_scale >= 0.f) || isinf(softmax_scale)) return KVR_ERR_INVALID_ARG;
+    if (sk->d.r != KVR_R) return KVR_ERR_UNSUPPORTED;          // the streaming side is written for r = 3
     LayerRange lr;
     kvr_status_t rc = layer_range(sk, layer, &lr);
     if (rc != KVR_OK) return rc;
@@ -408,6 +420,7 @@ kvr_status_t kvr_swap(kvr_sketch_t* sk, int32_t layer, void* Kr, void* Vr, int32
     if (!sk || !Kr || !Vr || !ret_idx || !row_scores) return KVR_ERR_INVALID_ARG;
     if (!aligned16(Kr) || !aligned16(Vr)) return KVR_ERR_INVALID_ARG;
     if (!(replace_rate > 0.f) || isinf(replace_rate) || max_swaps < 0) return KVR_ERR_INVALID_ARG;
+    if (sk->d.r != KVR_R) return KVR_ERR_UNSUPPORTED;          // the streaming side is written for r = 3
     LayerRange lr;
     kvr_status_t rc = layer_range(sk, layer, &lr);
     if (rc != KVR_OK) return rc;
@@ -429,6 +442,7 @@ kvr_status_t kvr_demote(kvr_sketch_t* sk, int32_t layer, const void* Kr, const v
     if (!sk || !Kr || !Vr || !ret_idx || !row_scores) return KVR_ERR_INVALID_ARG;
     if (!aligned16(Kr) || !aligned16(Vr) || !aligned16(Kr_out) || !aligned16(Vr_out)) return KVR_ERR_INVALID_ARG;
     if (Kr_out == Kr || Vr_out == Vr || ret_idx_out == ret_idx) return KVR_ERR_INVALID_ARG;
+    if (sk->d.r != KVR_R) return KVR_ERR_UNSUPPORTED;          // the streaming side is written for r = 3
     LayerRange lr;
     kvr_status_t rc = layer_range(sk, layer, &lr);
     if (rc != KVR_OK) return rc;
@@ -473,6 +487,7 @@ kvr_status_t kvr_append(kvr_sketch_t* sk, int32_t layer, const void* Kr, const v
         return KVR_ERR_INVALID_ARG;
     if (Kr_out == Kr || Vr_out == Vr || ret_idx_out == ret_idx || row_scores_out == row_scores) return KVR_ERR_INVALID_ARG;
     if (!(replace_rate > 0.f) || isinf(replace_rate) || max_swaps < 0) return KVR_ERR_INVALID_ARG;
+    if (sk->d.r != KVR_R) return KVR_ERR_UNSUPPORTED;          // the streaming side is written for r = 3
     LayerRange lr;
     kvr_status_t rc = layer_range(sk, layer, &lr);
     if (rc != KVR_OK) return rc;
@@ -629,7 +644,7 @@ kvr_status_t kvr_get_cells(const kvr_sketch_t* sk, int32_t layer, float* cells, 
     kvr_status_t rc = layer_range(sk, layer, &lr);
     if (rc != KVR_OK) return rc;
     DeviceGuard dg(sk->device);
-    const size_t per = (size_t)2 * KVR_R * sk->d.b * KVR_D;
+    const size_t per = (size_t)2 * sk->d.r * sk->d.b * KVR_D;
     KVR_CUDA(cudaMemcpyAsync(cells, sk->cells + (size_t)lr.inst0 * per, sizeof(float) * per * lr.n_inst,
                              cudaMemcpyDeviceToDevice, (cudaStream_t)cuda_stream));
     return KVR_OK;
@@ -647,7 +662,8 @@ kvr_status_t kvr_reconstruct(const kvr_sketch_t* sk, int32_t layer, float* Kt, f
     if (N == R) return KVR_OK;   // nothing was compressed: empty outputs
     if (!Kt && !Vt) return KVR_ERR_INVALID_ARG;
     DeviceGuard dg(sk->device);
-    KVR_CUDA(kvr_launch_reconstruct(sk, lr.inst0, lr.n_inst, N - R, Kt, Vt, (cudaStream_t)cuda_stream));
+    if (sk->d.r != KVR_R) KVR_CUDA(kvr_launch_reconstruct_generic(sk, lr.inst0, lr.n_inst, N - R, Kt, Vt, (cudaStream_t)cuda_stream));
+    else KVR_CUDA(kvr_launch_reconstruct(sk, lr.inst0, lr.n_inst, N - R, Kt, Vt, (cudaStream_t)cuda_stream));
     return KVR_OK;
 }
 

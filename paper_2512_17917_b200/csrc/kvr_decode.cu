@@ -341,6 +341,7 @@ extern "C" kvr_status_t kvr_decode_attention_static(kvr_sketch_t* sk, int32_t la
     auto misaligned = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
     if (misaligned(q) || misaligned(Kr) || misaligned(Vr) || misaligned(out)) return KVR_ERR_INVALID_ARG;
     if (!(softmax_scale >= 0.f) || isinf(softmax_scale)) return KVR_ERR_INVALID_ARG;
+    if (sk->d.r != KVR_R) return KVR_ERR_UNSUPPORTED;          // the split kernel behind this call is written for r = 3
     int inst0, n_inst, layer0, n_layers;
     if (layer == KVR_ALL_LAYERS) { inst0 = 0; n_inst = sk->n_inst; layer0 = 0; n_layers = sk->d.n_layers; }
     else if (layer >= 0 && layer < sk->d.n_layers) { inst0 = layer * sk->BH; n_inst = sk->BH; layer0 = layer; n_layers = 1; }

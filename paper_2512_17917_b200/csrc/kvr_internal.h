@@ -11,7 +11,8 @@
 #include "kvr.h"
 
 #define KVR_D 128       // head_dim the kernels are written for
-#define KVR_R 3         // sketch rows
+#define KVR_R 3         // sketch rows the fast kernels are written for (the paper's fixed value)
+#define KVR_R_MAX 5     // rows the general kernels accept (1, 3 or 5)
 #define KVR_HASH_P 2147483647ull
 
 // Per compressed token, packed for the decode kernels: bits 0-12 = cell of row 1, bits 13-25 =
@@ -152,6 +153,12 @@ cudaError_t kvr_launch_reconstruct(const kvr_sketch* sk, int inst0, int n_inst, 
                                    float* Vt, cudaStream_t st);
 cudaError_t kvr_launch_assignment(const kvr_sketch* sk, int inst0, int n_inst, int a, int32_t* cmp_idx,
                                   int32_t* bucket, int8_t* sign, cudaStream_t st);
+
+cudaError_t kvr_launch_decode_generic(kvr_sketch* sk, int inst0, int n_inst, int N, int R, int rows, const void* q,
+                                      const void* Kr, const void* Vr, float scale, float* out, int n_splits,
+                                      cudaStream_t st);
+cudaError_t kvr_launch_reconstruct_generic(const kvr_sketch* sk, int inst0, int n_inst, int a, float* Kt, float* Vt,
+                                           cudaStream_t st);
 
 int kvr_decode_staged_pick_C(int b, int G);
 bool kvr_decode_staged_plan(const kvr_sketch* sk, int n_inst, int N, int R, int rows, bool forced, KvrStagedPlan* plan);

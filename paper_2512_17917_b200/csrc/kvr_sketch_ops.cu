@@ -19,7 +19,7 @@ __global__ void __launch_bounds__(INS_THREADS)
 insert_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ full_list,
               const int8_t* __restrict__ tok_g, const uint32_t* __restrict__ bitmap_all, int bitmap_words,
               const uint2* __restrict__ K, const uint2* __restrict__ V, int N, int max_ctx, int b,
-              int inst0, int n_tbl, float* __restrict__ cells_all) {
+              int inst0, int n_tbl, int r, float* __restrict__ cells_all) {
     __shared__ uint32_t s_tok[INS_THREADS];
     __shared__ int s_wcnt[INS_THREADS / 32];
     __shared__ float4 s_part[2][KVR_D / 4];      // sums of the odd tokens: [keys | values][4 channels]
@@ -29,9 +29,9 @@ insert_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ 
     const int kv = warp & 1, par = warp >> 1;
     const uint32_t* bitmap = bitmap_all + (size_t)inst * bitmap_words;
     const int tb = n_tbl > 1 ? inst % n_tbl : 0;              // hash tables of this kv head (seeds per head) or the shared ones
-    full_off += (size_t)tb * KVR_R * (b + 1);
-    const int32_t* list = full_list + ((size_t)tb * KVR_R + i) * max_ctx;
-    const int8_t* g = tok_g + ((size_t)tb * KVR_R + i) * max_ctx;
+    full_off += (size_t)tb * r * (b + 1);
+    const int32_t* list = full_list + ((size_t)tb * r + i) * max_ctx;
+    const int8_t* g = tok_g + ((size_t)tb * r + i) * max_ctx;
     const uint2* src = (kv ? V : K) + (size_t)u * N * (KVR_D / 4) + lane;     // 4 channels (8 bytes) per lane
     const int p0 = full_off[i * (b + 1) + c], p1 = full_off[i * (b + 1) + c + 1];
 
@@ -102,7 +102,7 @@ insert_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ 
     __syncthreads();
     if (!par) {
         const float4 o = s_part[kv][lane];
-        float* cell = cells_all + ((((size_t)inst * 2 + kv) * KVR_R + i) * b + c) * KVR_D + 4 * lane;
+        float* cell = cells_all + ((((size_t)inst * 2 + kv) * r + i) * b + c) * KVR_D + 4 * lane;
         *reinterpret_cast<float4*>(cell) = make_float4(mine.x + o.x, mine.y + o.y, mine.z + o.z, mine.w + o.w);
     }
 }
@@ -144,16 +144,16 @@ __global__ void reconstruct_kernel(const float* __restrict__ cells_all, const in
 
 cudaError_t kvr_launch_insert(kvr_sketch* sk, int inst0, int n_inst, int N, const void* K, const void* V,
                               cudaStream_t st) {
-    dim3 g(sk->d.b, KVR_R, n_inst);
+    dim3 g(sk->d.b, sk->d.r, n_inst);
     if (sk->d.kv_dtype == KVR_F16)
         insert_kernel<__half><<<g, INS_THREADS, 0, st>>>(sk->full_off, sk->full_list, sk->tok_g, sk->bitmap,
                                                          sk->bitmap_words, (const uint2*)K, (const uint2*)V,
-                                                         N, sk->d.max_context, sk->d.b, inst0, sk->n_tbl, sk->cells);
+                                                         N, sk->d.max_context, sk->d.b, inst0, sk->n_tbl, sk->d.r, sk->cells);
     else
         insert_kernel<__nv_bfloat16><<<g, INS_THREADS, 0, st>>>(sk->full_off, sk->full_list, sk->tok_g, sk->bitmap,
                                                                 sk->bitmap_words, (const uint2*)K,
                                                                 (const uint2*)V, N, sk->d.max_context,
-                                                                sk->d.b, inst0, sk->n_tbl, sk->cells);
+                                                                sk->d.b, inst0, sk->n_tbl, sk->d.r, sk->cells);
     sk->launches += 1;
     return cudaGetLastError();
 }

@@ -14,7 +14,7 @@ namespace cg = cooperative_groups;
 namespace {
 
 struct SeedPack {
-    uint32_t s[KVR_R][4];
+    uint32_t s[KVR_R_MAX][4];
 };
 
 __device__ __forceinline__ uint32_t mix_index(uint32_t x, int mix) {
@@ -35,14 +35,15 @@ __device__ __forceinline__ uint32_t mod_p(uint64_t x) {
     return (uint32_t)y;
 }
 
-__global__ void hash_table_kernel(SeedPack sp, int mix, int b, int max_ctx, int32_t* __restrict__ tok_h,
+__global__ void hash_table_kernel(SeedPack sp, int r, int mix, int b, int max_ctx, int32_t* __restrict__ tok_h,
                                   int8_t* __restrict__ tok_g, uint32_t* __restrict__ tok_pack) {
     int J = blockIdx.x * blockDim.x + threadIdx.x;
     if (J >= max_ctx) return;
     uint64_t m = mix_index((uint32_t)J, mix);
-    uint32_t h[KVR_R], neg[KVR_R];
+    uint32_t h[KVR_R_MAX], neg[KVR_R_MAX];
 #pragma unroll
-    for (int i = 0; i < KVR_R; ++i) {
+    for (int i = 0; i < KVR_R_MAX; ++i) {
+        if (i >= r) { h[i] = 0; neg[i] = 0; continue; }
         uint32_t x = mod_p((uint64_t)sp.s[i][0] * m + sp.s[i][1]);
         h[i] = x % (uint32_t)b;
         uint32_t y = mod_p((uint64_t)sp.s[i][2] * m + sp.s[i][3]);
@@ -50,7 +51,7 @@ __global__ void hash_table_kernel(SeedPack sp, int mix, int b, int max_ctx, int3
         tok_h[(size_t)i * max_ctx + J] = (int32_t)h[i];
         tok_g[(size_t)i * max_ctx + J] = neg[i] ? (int8_t)-1 : (int8_t)1;
     }
-    tok_pack[J] = h[1] | (h[2] << KVR_PACK_H2_SHIFT) |
+    if (r == KVR_R) tok_pack[J] = h[1] | (h[2] << KVR_PACK_H2_SHIFT) |
                   ((neg[0] | (neg[1] << 1) | (neg[2] << 2)) << KVR_PACK_SIGN_SHIFT);
 }
 
@@ -292,44 +293,43 @@ lists_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ f
 }
 
 __global__ void assignment_kernel(const int32_t* __restrict__ cmp_all, const int32_t* __restrict__ tok_h,
-                                  const int8_t* __restrict__ tok_g, int max_ctx, int a, int inst0, int n_tbl,
+                                  const int8_t* __restrict__ tok_g, int r, int max_ctx, int a, int inst0, int n_tbl,
                                   int32_t* __restrict__ cmp_out, int32_t* __restrict__ bucket,
                                   int8_t* __restrict__ sign) {
     int t = blockIdx.x * blockDim.x + threadIdx.x;
     int u = blockIdx.y;
     if (t >= a) return;
     const int tb = n_tbl > 1 ? (inst0 + u) % n_tbl : 0;
-    tok_h += (size_t)tb * KVR_R * max_ctx;
-    tok_g += (size_t)tb * KVR_R * max_ctx;
+    tok_h += (size_t)tb * r * max_ctx;
+    tok_g += (size_t)tb * r * max_ctx;
     int J = cmp_all[(size_t)(inst0 + u) * max_ctx + t];
     if (cmp_out) cmp_out[(size_t)u * a + t] = J;
-#pragma unroll
-    for (int i = 0; i < KVR_R; ++i) {
-        if (bucket) bucket[((size_t)u * KVR_R + i) * a + t] = tok_h[(size_t)i * max_ctx + J];
-        if (sign) sign[((size_t)u * KVR_R + i) * a + t] = tok_g[(size_t)i * max_ctx + J];
+    for (int i = 0; i < r; ++i) {
+        if (bucket) bucket[((size_t)u * r + i) * a + t] = tok_h[(size_t)i * max_ctx + J];
+        if (sign) sign[((size_t)u * r + i) * a + t] = tok_g[(size_t)i * max_ctx + J];
     }
 }
 
 }  // namespace
 
 cudaError_t kvr_launch_hash_tables(kvr_sketch* sk, cudaStream_t st) {
-    const int b = sk->d.b, mc = sk->d.max_context;
+    const int b = sk->d.b, mc = sk->d.max_context, r = sk->d.r;
     int32_t* cnt = nullptr;
-    cudaError_t e = cudaMalloc(&cnt, sizeof(int32_t) * KVR_R * b);
+    cudaError_t e = cudaMalloc(&cnt, sizeof(int32_t) * r * b);
     if (e != cudaSuccess) return e;
     for (int t = 0; t < sk->n_tbl; ++t) {                       // one set of tables per kv head, or one for all
-        SeedPack sp;
-        for (int i = 0; i < KVR_R; ++i)
-            for (int k = 0; k < 4; ++k) sp.s[i][k] = sk->seeds[((size_t)t * KVR_R + i) * 4 + k];
-        int32_t* tok_h = sk->tok_h + (size_t)t * KVR_R * mc;
-        int8_t* tok_g = sk->tok_g + (size_t)t * KVR_R * mc;
-        int32_t* full_off = sk->full_off + (size_t)t * KVR_R * (b + 1);
-        int32_t* full_list = sk->full_list + (size_t)t * KVR_R * mc;
-        hash_table_kernel<<<(mc + 255) / 256, 256, 0, st>>>(sp, sk->d.index_mix, b, mc, tok_h, tok_g,
+        SeedPack sp = {};
+        for (int i = 0; i < r; ++i)
+            for (int k = 0; k < 4; ++k) sp.s[i][k] = sk->seeds[((size_t)t * r + i) * 4 + k];
+        int32_t* tok_h = sk->tok_h + (size_t)t * r * mc;
+        int8_t* tok_g = sk->tok_g + (size_t)t * r * mc;
+        int32_t* full_off = sk->full_off + (size_t)t * r * (b + 1);
+        int32_t* full_list = sk->full_list + (size_t)t * r * mc;
+        hash_table_kernel<<<(mc + 255) / 256, 256, 0, st>>>(sp, r, sk->d.index_mix, b, mc, tok_h, tok_g,
                                                             sk->tok_pack + (size_t)t * mc);
-        dim3 g((b + 127) / 128, KVR_R);
+        dim3 g((b + 127) / 128, r);
         csr_count_kernel<<<g, 128, 0, st>>>(tok_h, b, mc, cnt);
-        csr_scan_kernel<<<KVR_R, 1024, 0, st>>>(cnt, b, full_off);
+        csr_scan_kernel<<<r, 1024, 0, st>>>(cnt, b, full_off);
         csr_fill_kernel<<<g, 128, 0, st>>>(tok_h, full_off, b, mc, full_list);
         sk->launches += 4;
     }
@@ -356,7 +356,7 @@ cudaError_t kvr_launch_assignment(const kvr_sketch* sk, int inst0, int n_inst, i
                                   int32_t* bucket, int8_t* sign, cudaStream_t st) {
     if (a <= 0 || n_inst <= 0) return cudaSuccess;
     dim3 g((a + 255) / 256, n_inst);
-    assignment_kernel<<<g, 256, 0, st>>>(sk->cmp_idx, sk->tok_h, sk->tok_g, sk->d.max_context, a, inst0, sk->n_tbl,
+    assignment_kernel<<<g, 256, 0, st>>>(sk->cmp_idx, sk->tok_h, sk->tok_g, sk->d.r, sk->d.max_context, a, inst0, sk->n_tbl,
                                          cmp_idx, bucket, sign);
     const_cast<kvr_sketch*>(sk)->launches += 1;
     return cudaGetLastError();

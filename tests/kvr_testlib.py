@@ -93,8 +93,9 @@ def run_and_check(K, V, Qobs, q, *, R, n_recent, b, seeds, index_mix=True, layer
     L, B, H, N, D = K.shape
     Hq, W = Qobs.shape[2], Qobs.shape[3]
     G = Hq // H
+    r = int(np.asarray(seeds).shape[0])                      # sketch rows = sets of (A, C, A', C')
     dev = "cuda"
-    sk = kvr.kvr_sketch_create(b=b, batch=B, n_layers=L, n_kv_heads=H, n_q_heads=Hq, max_context=N,
+    sk = kvr.kvr_sketch_create(b=b, batch=B, n_layers=L, n_kv_heads=H, n_q_heads=Hq, max_context=N, r=r,
                                kv_dtype=K.dtype, hash_seeds=seeds, index_mix=index_mix, device=dev)
     if decode_kernel is not None:
         kvr.kvr_sketch_set_decode_kernel(sk, decode_kernel)
@@ -154,14 +155,14 @@ def run_and_check(K, V, Qobs, q, *, R, n_recent, b, seeds, index_mix=True, layer
     assert (Kr_g == orc.gather(Kc, ret_g)).all() and (Vr_g == orc.gather(Vc, ret_g)).all()
     # --- hashing -------------------------------------------------------------------------------
     if a:
-        bk = bucket_gpu.reshape(n_inst, 3, a).cpu().numpy()[sel]
-        sg = sign_gpu.reshape(n_inst, 3, a).cpu().numpy()[sel]
+        bk = bucket_gpu.reshape(n_inst, r, a).cpu().numpy()[sel]
+        sg = sign_gpu.reshape(n_inst, r, a).cpu().numpy()[sel]
         for u in range(len(sel)):
             bo, so = orc.bucket_sign(cmp_g[u], seeds, b, mix=index_mix)
             assert (bk[u] == bo).all() and (sg[u] == so).all(), "bucket / sign assignment"
     # --- cells (oracle re-run on the kernel's selection) -----------------------------------------
     cells_o = orc.insert(Kc, Vc, cmp_g, seeds, b, mix=index_mix)              # [n, r, b, 2, D]
-    cells_g = cells_gpu.reshape(n_inst, 2, 3, b, D).cpu().numpy()[sel].transpose(0, 2, 3, 1, 4)
+    cells_g = cells_gpu.reshape(n_inst, 2, r, b, D).cpu().numpy()[sel].transpose(0, 2, 3, 1, 4)
     assert np.abs(cells_g - cells_o).max() <= TOL, np.abs(cells_g - cells_o).max()
     # --- reconstruction ------------------------------------------------------------------------
     if check_reconstruct and a:

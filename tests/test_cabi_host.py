@@ -50,7 +50,7 @@ def _create(**over):
 @pytest.mark.parametrize("over,status", [
     (dict(b=0), 1), (dict(batch=0), 1), (dict(max_context=0), 1), (dict(kv_dtype=7), 1),
     (dict(n_q_heads=7), 1), (dict(index_mix=2), 1), (dict(seeds_per_head=2), 1),
-    (dict(r=5), 2), (dict(head_dim=64), 2), (dict(b=8193), 2), (dict(n_q_heads=6), 2),
+    (dict(r=7), 2), (dict(r=2), 2), (dict(head_dim=64), 2), (dict(b=8193), 2), (dict(n_q_heads=6), 2),
     (dict(batch=4096, n_layers=64), 2),
 ])
 def test_create_rejects_bad_descriptors_without_a_device(over, status):

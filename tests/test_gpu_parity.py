@@ -564,6 +564,50 @@ def test_hash_seeds_per_kv_head(which):
     kvr.kvr_sketch_destroy(sk)
 
 
+@pytest.mark.parametrize("r,dtype,Hq,combine", [(1, F16, 8, "median"), (5, F16, 8, "median"), (5, BF16, 16, "median"),
+                                               (5, F16, 4, "mean"), (1, BF16, 2, "median")])
+def test_sketches_with_one_and_five_rows(r, dtype, Hq, combine):
+    """r = 1 (Algorithm 2 is a direct look-up) and r = 5 (middle of five): hashing, cells,
+    reconstruction and decode against the oracle, which is generic in r; 1 to 8 query heads per kv
+    head, the mean combine, two layers in one call."""
+    B, H, L, N, W, R, b = 1, 2, 2, 1300, 8, 140, 17
+    K, V, Q, q = make_case(8100 + r, B, H, Hq, N, W, dtype, L)
+    seeds = synth.hash_seeds(8200 + r, r=r)
+    run_and_check(K, V, Q, q, R=R, n_recent=7, b=b, seeds=seeds, layer_mode="all", combine=combine)
+
+
+def test_one_row_sketch_without_collisions_is_the_full_cache():
+    """r = 1 with one cell per token (raw indices, h(J) = J): every vague token is looked up exactly,
+    so the decode equals attention over the uncompressed cache."""
+    B, H, Hq, N, W, R = 1, 2, 8, 500, 4, 50
+    K, V, Q, q = make_case(8300, B, H, Hq, N, W, F16, 1)
+    seeds = synth.injective_seeds()[:1]
+    out_g, out_o = run_and_check(K, V, Q, q, R=R, n_recent=0, b=N, seeds=seeds, index_mix=False)
+    G = Hq // H
+    Kc, Vc, qc = inst_major(K[0]).astype(np.float64), inst_major(V[0]).astype(np.float64), dec_to_inst(q[0], H).astype(np.float64)
+    logits = np.einsum("ugd,ujd->ugj", qc, Kc) / math.sqrt(128)
+    p = np.exp(logits - logits.max(-1, keepdims=True))
+    full = np.einsum("ugj,ujd->ugd", p / p.sum(-1, keepdims=True), Vc)
+    assert np.abs(out_g - full).max() <= TOL
+
+
+def test_calls_written_for_three_rows_say_so():
+    """The streaming side, the multi-query call and the allocation-free call serve r = 3 only."""
+    K, V, Q, q = make_case(8400, 1, 2, 8, 300, 4, F16, 1)
+    sk = kvr.kvr_sketch_create(b=9, batch=1, n_layers=1, n_kv_heads=2, n_q_heads=8, max_context=300, r=5, kv_dtype=F16,
+                               hash_seeds=synth.hash_seeds(8401, r=5))
+    Kr, Vr, ret = kvr.kvr_compress(sk, 0, K[0].cuda(), V[0].cuda(), Q[0].cuda(), 30, 0)
+    qd = q[0].cuda()
+    kvr.kvr_decode_attention(sk, 0, qd, Kr, Vr, ret)
+    for call in (lambda: kvr.kvr_accumulate_vague_scores(sk, 0, qd),
+                 lambda: kvr.kvr_decode_attention_static(sk, 0, qd, Kr, Vr, ret),
+                 lambda: kvr.kvr_decode_attention_mq(sk, 0, torch.zeros((1, 8, 2, 128), dtype=F16, device="cuda"), Kr, Vr, ret)):
+        with pytest.raises(kvr.KvrError) as e:
+            call()
+        assert e.value.status == 2
+    kvr.kvr_sketch_destroy(sk)
+
+
 def test_per_layer_budgets_in_one_handle():
     """Budgets that differ from layer to layer (kvr_layer_budgets from per-layer weights): every layer
     of one handle is compressed with its own budget and decoded; selection, cells and outputs against
