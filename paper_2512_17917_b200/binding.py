@@ -32,7 +32,7 @@ EXPORTS = (
     "kvr_sketch_set_decode_kernel", "kvr_last_decode_kernel", "kvr_sketch_device_status",
     "kvr_accumulate_scores", "kvr_demote", "kvr_sketch_set_score_kernel", "kvr_last_score_kernel",
     "kvr_accumulate_vague_scores", "kvr_swap", "kvr_sketch_set_obs_window_causal", "kvr_paper_storage_split", "kvr_layer_budgets", "kvr_sketch_set_combine",
-    "kvr_measure_pipe_peaks", "kvr_append", "kvr_append_sizes", "kvr_decode_attention_mq",
+    "kvr_measure_pipe_peaks", "kvr_append", "kvr_append_sizes", "kvr_decode_attention_mq", "kvr_sketch_set_wait_test",
 )
 
 
@@ -96,6 +96,7 @@ def lib() -> ctypes.CDLL:
         L.kvr_last_decode_kernel.argtypes = [vp]
         L.kvr_last_decode_kernel.restype = i32
         L.kvr_decode_attention_mq.argtypes = [vp, i32, vp, vp, vp, vp, i32, i32, i32, f32, vp, vp]
+        L.kvr_sketch_set_wait_test.argtypes = [vp, ctypes.c_int64, i32]
         L.kvr_append_sizes.argtypes = [i32, i32, i32, i32, i32, i32, ctypes.POINTER(i32)]
         L.kvr_append_sizes.restype = i32
         L.kvr_append.argtypes = [vp, i32, vp, vp, vp, vp, i32, i32, vp, vp, i32, i32, i32, i32, f32, i32, vp, vp, vp, vp, vp, vp]
@@ -245,6 +246,10 @@ def kvr_measure_pipe_peaks(stream=None):
     out = (ctypes.c_double * 2)()
     _check(lib().kvr_measure_pipe_peaks(out, _stream(stream)), "kvr_measure_pipe_peaks")
     return float(out[0]), float(out[1])
+
+
+def kvr_sketch_set_wait_test(sk: Sketch, wait_limit_ns: int, unannounced_bytes: int):
+    _check(lib().kvr_sketch_set_wait_test(sk.handle, int(wait_limit_ns), int(unannounced_bytes)), "kvr_sketch_set_wait_test")
 
 
 def kvr_launch_count(sk: Sketch) -> int:

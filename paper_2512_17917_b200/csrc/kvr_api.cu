@@ -231,6 +231,8 @@ kvr_status_t kvr_sketch_create(kvr_sketch_t** out, const kvr_sketch_desc_t* desc
     while ((1 << sk->logC) < sk->C) ++sk->logC;
     sk->n1 = sk->C > 0 ? (d.b + sk->C - 1) / sk->C : 0;
     sk->decode_kernel = KVR_DECODE_AUTO;
+    sk->wait_ns = 200ull * 1000 * 1000;
+    sk->tx_extra = 0;
     sk->last_decode_kernel = KVR_DECODE_AUTO;
     sk->score_kernel = KVR_SCORE_AUTO;
     sk->obs_causal = 0;
@@ -680,6 +682,16 @@ kvr_status_t kvr_sketch_device_status(kvr_sketch_t* sk, int32_t* status, void* c
     cudaStream_t st = (cudaStream_t)cuda_stream;
     KVR_CUDA(cudaMemcpyAsync(status, sk->dev_status, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     KVR_CUDA(cudaStreamSynchronize(st));
+    return KVR_OK;
+}
+
+kvr_status_t kvr_sketch_set_wait_test(kvr_sketch_t* sk, int64_t wait_limit_ns, int32_t unannounced_bytes) {
+    if (!sk) return KVR_ERR_INVALID_ARG;
+    // the copies land within microseconds: a limit of 100 us or more never cuts a copy short
+    if (wait_limit_ns < 100 * 1000 || wait_limit_ns > 1000ll * 1000 * 1000) return KVR_ERR_INVALID_ARG;
+    if (unannounced_bytes < 0 || unannounced_bytes > 4096 || (unannounced_bytes & 15)) return KVR_ERR_INVALID_ARG;
+    sk->wait_ns = (unsigned long long)wait_limit_ns;
+    sk->tx_extra = (uint32_t)unannounced_bytes;
     return KVR_OK;
 }
 

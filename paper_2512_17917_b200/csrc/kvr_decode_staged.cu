@@ -74,6 +74,8 @@ struct StagedParams {
     int lcap;               // token entries staged at a time
     int rcap, rcap_extra;   // retained rows whose logits fit beside them (class CTAs / row-only CTAs)
     int n_ccta, r_cls;      // class CTAs per head-instance; retained rows they share (extra CTAs take the rest)
+    unsigned long long wait_ns;   // how long a wait on a staging barrier may last (200 ms unless a test shortens it)
+    uint32_t tx_extra;      // 0; a test announces more bytes than are copied, so that the cells barrier never completes
     uint32_t zero;          // 0, unknown to the compiler (orders a shared-memory read before a copy into the same bytes)
     float scale_log2e;
 };
@@ -133,16 +135,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: the copies this kernel waits for take microseconds; a wait that lasts WAIT_LIMIT_NS
+// Bounded wait: the copies this kernel waits for take microseconds; a wait that lasts limit_ns
 // gives up (the caller records it in the handle's status word) instead of hanging the GPU.
-constexpr unsigned long long WAIT_LIMIT_NS = 200ull * 1000 * 1000;
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     unsigned long long t0, t;
     asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t0));
     while (!mbar_try_wait(bar, parity)) {
         asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t));
-        if (t - t0 > WAIT_LIMIT_NS) return false;
+        if (t - t0 > limit_ns) return false;
     }
     return true;
 }
@@ -260,7 +261,7 @@ decode_staged_kernel(const StagedParams p) {
             mbar_init(bar_cells, 1);
             mbar_init(bar_list, 1);
             const int cnt1 = (b - ci + C - 1) >> p.logC, cnt2 = (b - cj + C - 1) >> p.logC;   // cells of the two slices
-            mbar_expect_tx(bar_cells, (uint32_t)((cnt1 + cnt2) * CELLB));
+            mbar_expect_tx(bar_cells, (uint32_t)((cnt1 + cnt2) * CELLB) + p.tx_extra);
         }
         __syncthreads();
         for (int i = warp + lane * NW; i < 4 * n1; i += NT) {       // one 512-byte piece per (cell, keys | values)
@@ -459,7 +460,7 @@ decode_staged_kernel(const StagedParams p) {
         // weight slot, w = row-0 cell of the next run << 16 | address of its sign pairs | run flag
         // (also set for the first token of every group).  The entries lie in the upper half of the
         // descriptor array; a batch of descriptors only overwrites entries that were read before.
-        if (st == 0 && len0 > 0 && !mbar_wait(bar_list, 0)) atomicOr(p.status, 1);       // the first entries have landed
+        if (st == 0 && len0 > 0 && !mbar_wait(bar_list, 0, p.wait_ns)) atomicOr(p.status, 1);       // the first entries have landed
         const float* g0K = p.cells + (size_t)inst * 2 * KVR_R * b * KVR_D + 4 * lg;      // this lane's piece of row-0 cell 0, key half
         {
             const uint2* staged = reinterpret_cast<const uint2*>(smem + L.stage) + lshift;
@@ -497,7 +498,7 @@ decode_staged_kernel(const StagedParams p) {
             }
             __syncthreads();
         }
-        if (st == 0 && !extra && !mbar_wait(bar_cells, 0)) atomicOr(p.status, 1);       // the cells have landed
+        if (st == 0 && !extra && !mbar_wait(bar_cells, 0, p.wait_ns)) atomicOr(p.status, 1);       // the cells have landed
         // compressed tokens (Algorithm 2 on the key halves)
         if (len > 0) {
             float k0[DPL];                                // key half of the run's row-0 cell (this lane's channels)
@@ -871,6 +872,8 @@ cudaError_t kvr_launch_decode_staged(kvr_sketch* sk, int inst0, int n_inst, int 
     p.n_ccta = plan.records - plan.extra;
     p.r_cls = plan.r_cls;
     p.zero = 0u;
+    p.wait_ns = sk->wait_ns;
+    p.tx_extra = sk->tx_extra;
     p.scale_log2e = scale * 1.4426950408889634f;
     sk->launches += 1;
     const bool f16 = sk->d.kv_dtype == KVR_F16;

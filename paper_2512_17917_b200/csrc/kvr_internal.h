@@ -87,6 +87,8 @@ struct kvr_sketch {
     // ---- decode kernel choice ----
     int decode_kernel;       // kvr_decode_kernel_t requested by the caller
     int last_decode_kernel;  // which kernel the last decode call launched (KVR_DECODE_SPLIT / _STAGED)
+    unsigned long long wait_ns;   // limit of the staged decode kernel's waits on its staging barriers
+    uint32_t tx_extra;       // bytes the staged kernel announces beyond what it copies (test hook; 0)
     int score_kernel;        // kvr_score_kernel_t requested by the caller
     int obs_causal;          // observation window inside the context, causally masked
     int combine;             // kvr_combine_t: 0 = element-wise median of the three cells, 1 = their mean

@@ -608,6 +608,39 @@ def test_calls_written_for_three_rows_say_so():
     kvr.kvr_sketch_destroy(sk)
 
 
+def test_bounded_wait_gives_up_and_reports():
+    """The staged kernel's wait on its staging barrier is bounded.  With the test hook the kernel expects
+    more bytes than its copies deliver, so the barrier never completes: every class CTA waits the
+    (shortened) limit, sets the status bit and carries on; the cells had landed long before, so the
+    output still matches an untouched handle.  Nothing faults or hangs; normal operation afterwards."""
+    seeds = synth.hash_seeds(9100)
+    K, V, Q, q = make_case(9101, 1, 2, 8, 2000, 8, F16, 1)
+    dev = "cuda"
+    outs = []
+    for hook in (False, True):
+        sk = kvr.kvr_sketch_create(b=25, batch=1, n_layers=1, n_kv_heads=2, n_q_heads=8, max_context=2000, kv_dtype=F16,
+                                   hash_seeds=seeds)
+        kvr.kvr_sketch_set_decode_kernel(sk, kvr.KVR_DECODE_STAGED)
+        Kr, Vr, ret = kvr.kvr_compress(sk, 0, K[0].to(dev), V[0].to(dev), Q[0].to(dev), 200, 0)
+        if hook:
+            kvr.kvr_sketch_set_wait_test(sk, 1_000_000, 16)                     # 1 ms, 16 bytes that never arrive
+        outs.append(kvr.kvr_decode_attention(sk, 0, q[0].to(dev), Kr, Vr, ret).clone())
+        assert kvr.kvr_sketch_device_status(sk) == (1 if hook else 0)
+        if hook:
+            kvr.kvr_sketch_set_wait_test(sk, 200_000_000, 0)
+            again = kvr.kvr_decode_attention(sk, 0, q[0].to(dev), Kr, Vr, ret)
+            assert torch.equal(again, outs[0])
+        kvr.kvr_sketch_destroy(sk)
+    assert torch.equal(outs[0], outs[1])
+    with pytest.raises(kvr.KvrError):
+        sk = kvr.kvr_sketch_create(b=5, batch=1, n_layers=1, n_kv_heads=1, n_q_heads=1, max_context=64, kv_dtype=F16,
+                                   hash_seeds=seeds)
+        try:
+            kvr.kvr_sketch_set_wait_test(sk, 10, 16)                            # a limit that could cut a copy short
+        finally:
+            kvr.kvr_sketch_destroy(sk)
+
+
 def test_per_layer_budgets_in_one_handle():
     """Budgets that differ from layer to layer (kvr_layer_budgets from per-layer weights): every layer
     of one handle is compressed with its own budget and decoded; selection, cells and outputs against
