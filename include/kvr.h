@@ -211,6 +211,19 @@ kvr_status_t kvr_accumulate_scores(kvr_sketch_t* sk, int32_t layer, const void* 
                                    int32_t n_rows, float softmax_scale, float* score_acc,
                                    void* cuda_stream);
 
+/* kvr_decode_attention, kvr_accumulate_scores and kvr_accumulate_vague_scores as one call: the paper's
+ * Calculation Phase keeps the attention scores of the step it has just computed (Overview), it does not
+ * compute them twice.  Arguments as kvr_decode_attention plus score_acc [batch, n_kv_heads, n_retained]
+ * float32, in/out (as in kvr_accumulate_scores).  Where the staged decode kernel serves the call it writes
+ * every logit it computes to a workspace of the handle ((n_retained + compressed tokens) x query heads per
+ * kv head x 4 bytes per head-instance, allocated on first use) and one small kernel turns them into mass:
+ * the cache is read once.  Where the split kernel serves it, the two accumulate kernels run after it.
+ * Both give the same sums up to the order of fp32 additions inside a logit.
+ * Errors: as kvr_decode_attention, ALLOC, UNSUPPORTED for r != 3. */
+kvr_status_t kvr_decode_attention_scored(kvr_sketch_t* sk, int32_t layer, const void* q, const void* Kr,
+                                         const void* Vr, const int32_t* ret_idx, int32_t n_retained,
+                                         float softmax_scale, float* out, float* score_acc, void* cuda_stream);
+
 /* Overflow step.  Kr, Vr [batch, n_kv_heads, n_rows, head_dim] and ret_idx [.., n_rows] (ascending
  * token indices: the retained tokens of the compress followed by the appended ones) hold more than
  * `budget` rows.  Per head-instance the newest n_recent rows stay (Recent part), the budget - n_recent

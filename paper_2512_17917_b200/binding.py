@@ -32,7 +32,7 @@ EXPORTS = (
     "kvr_sketch_set_decode_kernel", "kvr_last_decode_kernel", "kvr_sketch_device_status",
     "kvr_accumulate_scores", "kvr_demote", "kvr_sketch_set_score_kernel", "kvr_last_score_kernel",
     "kvr_accumulate_vague_scores", "kvr_swap", "kvr_sketch_set_obs_window_causal", "kvr_paper_storage_split", "kvr_layer_budgets", "kvr_sketch_set_combine",
-    "kvr_measure_pipe_peaks", "kvr_append", "kvr_append_sizes", "kvr_decode_attention_mq", "kvr_sketch_set_wait_test",
+    "kvr_measure_pipe_peaks", "kvr_append", "kvr_append_sizes", "kvr_decode_attention_mq", "kvr_sketch_set_wait_test", "kvr_decode_attention_scored",
 )
 
 
@@ -71,6 +71,7 @@ def lib() -> ctypes.CDLL:
         L.kvr_compress.argtypes = [vp, i32, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp]
         L.kvr_decode_attention.argtypes = [vp, i32, vp, vp, vp, vp, i32, f32, vp, vp]
         L.kvr_decode_attention_static.argtypes = [vp, i32, vp, vp, vp, vp, i32, f32, vp, vp]
+        L.kvr_decode_attention_scored.argtypes = [vp, i32, vp, vp, vp, vp, i32, f32, vp, vp, vp]
         L.kvr_compress_host.argtypes = [vp, i32, vp, vp, vp, i32, i32, i32, i32, vp]
         L.kvr_decode_attention_host.argtypes = [vp, i32, vp, f32, vp, vp]
         L.kvr_get_scores.argtypes = [vp, i32, vp, vp]
@@ -298,6 +299,25 @@ def kvr_decode_attention(sk: Sketch, layer: int, q, Kr, Vr, ret_idx, *, softmax_
                                     _ptr(ret_idx) if R else None, R, float(softmax_scale), _ptr(out),
                                     _stream(stream))
     _check(st, "kvr_decode_attention")
+    return out
+
+
+def kvr_decode_attention_scored(sk: Sketch, layer: int, q, Kr, Vr, ret_idx, score_acc, *, softmax_scale: float = 0.0,
+                                out=None, stream=None):
+    """kvr_decode_attention_scored: the decode call that also adds the step's attention mass to score_acc
+    [.., H, n_rows] (float32, in place) and to the handle's per-token scores of the vague tokens."""
+    d = sk.desc
+    lead = _lead(sk, layer)
+    assert tuple(q.shape) == lead + (d.n_q_heads, d.head_dim) and q.dtype == sk.torch_dtype, "q shape/dtype"
+    R = Kr.shape[-2]
+    assert score_acc.dtype == torch.float32 and score_acc.shape[-1] == R and score_acc.is_contiguous()
+    if out is None:
+        out = torch.empty(lead + (d.n_q_heads, d.head_dim), dtype=torch.float32, device=q.device)
+    with torch.cuda.device(sk.device):
+        st = lib().kvr_decode_attention_scored(sk.handle, layer, _ptr(q), _ptr(Kr) if R else None, _ptr(Vr) if R else None,
+                                               _ptr(ret_idx) if R else None, R, float(softmax_scale), _ptr(out),
+                                               _ptr(score_acc), _stream(stream))
+    _check(st, "kvr_decode_attention_scored")
     return out
 
 

@@ -48,7 +48,7 @@ kvr_status_t ensure(kvr_sketch* sk, void** p, size_t* cur, size_t need) {
 
 void free_all(kvr_sketch* sk) {
     void* ptrs[] = {sk->tok_h, sk->tok_g, sk->tok_pack, sk->full_off, sk->full_list, sk->cells, sk->scores,
-                    sk->cmp_idx, sk->bitmap, sk->dlist, sk->doff, sk->ws_score, sk->ws_decode, sk->tickets, sk->clist, sk->coff, sk->dev_status, sk->ml, sk->ws_demote, sk->ws_append,
+                    sk->cmp_idx, sk->bitmap, sk->dlist, sk->doff, sk->ws_score, sk->ws_decode, sk->tickets, sk->clist, sk->coff, sk->ctok, sk->dev_status, sk->ml, sk->ws_demote, sk->ws_append, sk->ws_emit,
                     sk->st_K, sk->st_V, sk->st_Q, sk->st_Kr, sk->st_Vr, sk->st_ret, sk->st_q1, sk->st_out};
     for (void* p : ptrs)
         if (p) cudaFree(p);
@@ -146,8 +146,10 @@ kvr_status_t compress_impl(kvr_sketch* sk, const LayerRange& lr, const void* K, 
     return KVR_OK;
 }
 
+// score_acc (or null): also add this call's attention mass to the rows' scores (score_acc) and to the
+// vague tokens' scores (the handle's per-token array).
 kvr_status_t decode_impl(kvr_sketch* sk, const LayerRange& lr, int N, int R, int rows, const void* q, const void* Kr,
-                         const void* Vr, float scale, float* out, cudaStream_t st) {
+                         const void* Vr, float scale, float* out, cudaStream_t st, float* score_acc = nullptr) {
     if (scale == 0.f) scale = (float)(1.0 / sqrt((double)sk->d.head_dim));
     if (sk->d.r != KVR_R) {                        // r = 1 or 5: the general kernel
         if (sk->decode_kernel == KVR_DECODE_STAGED) return KVR_ERR_UNSUPPORTED;
@@ -165,9 +167,17 @@ kvr_status_t decode_impl(kvr_sketch* sk, const LayerRange& lr, int N, int R, int
         kvr_status_t rc = ensure(sk, &sk->ws_decode, &sk->ws_decode_bytes,
                                  kvr_decode_ws_bytes(lr.n_inst, plan.records, sk->G));
         if (rc != KVR_OK) return rc;
+        float* emit = nullptr;
+        if (score_acc) {                           // the kernel hands out its logits: no second pass over the cache
+            rc = ensure(sk, &sk->ws_emit, &sk->ws_emit_bytes,
+                        sizeof(float) * (size_t)lr.n_inst * (size_t)(rows + N - R) * sk->G + 16);
+            if (rc != KVR_OK) return rc;
+            emit = (float*)sk->ws_emit;
+        }
         KVR_CUDA(kvr_launch_decode_staged(sk, lr.inst0, lr.n_inst, N, R, rows, q, Kr, Vr, scale, out, plan,
-                                          (float*)sk->ws_decode, sk->tickets, st));
+                                          (float*)sk->ws_decode, sk->tickets, emit, st));
         sk->last_decode_kernel = KVR_DECODE_STAGED;
+        if (emit) KVR_CUDA(kvr_launch_apply_emitted(sk, lr.inst0, lr.n_inst, rows, N - R, emit, score_acc, st));
         return KVR_OK;
     }
     const int S = kvr_decode_pick_splits(sk, lr.n_inst, N, R);
@@ -175,6 +185,10 @@ kvr_status_t decode_impl(kvr_sketch* sk, const LayerRange& lr, int N, int R, int
     if (rc != KVR_OK) return rc;
     KVR_CUDA(kvr_launch_decode(sk, lr.inst0, lr.n_inst, N, R, rows, q, Kr, Vr, scale, out, S, st));
     sk->last_decode_kernel = KVR_DECODE_SPLIT;
+    if (score_acc) {                               // the split kernel keeps no logits: a second pass computes them again
+        KVR_CUDA(kvr_launch_row_mass(sk, lr.inst0, lr.n_inst, rows, q, Kr, scale, score_acc, st));
+        KVR_CUDA(kvr_launch_vague_mass(sk, lr.inst0, lr.n_inst, N - R, q, scale, st));
+    }
     return KVR_OK;
 }
 
@@ -270,6 +284,7 @@ kvr_status_t kvr_sketch_create(kvr_sketch_t** out, const kvr_sketch_desc_t* desc
     if (sk->C > 0) {
         A(&sk->clist, sizeof(uint2) * (ni * mc + 2));     // +2: the staged kernel copies whole 16-byte pairs
         A(&sk->coff, sizeof(int32_t) * ni * (sk->C * sk->C + 1));
+        A(&sk->ctok, sizeof(int32_t) * ni * mc);
     }
     if (rc != KVR_OK) { free_all(sk); delete sk; return rc; }
     cudaError_t e = cudaMemsetAsync(sk->cells, 0, cell_bytes, st);
@@ -348,6 +363,26 @@ kvr_status_t kvr_decode_attention(kvr_sketch_t* sk, int32_t layer, const void* q
     if (n_retained > 0 && (!Kr || !Vr)) return KVR_ERR_INVALID_ARG;
     DeviceGuard dg(sk->device);
     return decode_impl(sk, lr, N, R, n_retained, q, Kr, Vr, softmax_scale, out, (cudaStream_t)cuda_stream);
+}
+
+kvr_status_t kvr_decode_attention_scored(kvr_sketch_t* sk, int32_t layer, const void* q, const void* Kr, const void* Vr,
+                                         const int32_t* ret_idx, int32_t n_retained, float softmax_scale, float* out,
+                                         float* score_acc, void* cuda_stream) {
+    (void)ret_idx;
+    if (!sk || !q || !out || !score_acc) return KVR_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(Kr) || !aligned16(Vr) || !aligned16(out)) return KVR_ERR_INVALID_ARG;
+    if (!(softmax_scale >= 0.f) || isinf(softmax_scale)) return KVR_ERR_INVALID_ARG;
+    if (sk->d.r != KVR_R) return KVR_ERR_UNSUPPORTED;          // the streaming side is written for r = 3
+    LayerRange lr;
+    kvr_status_t rc = layer_range(sk, layer, &lr);
+    if (rc != KVR_OK) return rc;
+    int N, R;
+    rc = layer_state(sk, lr, &N, &R);
+    if (rc != KVR_OK) return rc;
+    if (n_retained < R) return KVR_ERR_SHAPE;
+    if (n_retained > 0 && (!Kr || !Vr)) return KVR_ERR_INVALID_ARG;
+    DeviceGuard dg(sk->device);
+    return decode_impl(sk, lr, N, R, n_retained, q, Kr, Vr, softmax_scale, out, (cudaStream_t)cuda_stream, score_acc);
 }
 
 kvr_status_t kvr_decode_attention_mq(kvr_sketch_t* sk, int32_t layer, const void* q, const void* Kr, const void* Vr,

@@ -74,6 +74,8 @@ struct StagedParams {
     int lcap;               // token entries staged at a time
     int rcap, rcap_extra;   // retained rows whose logits fit beside them (class CTAs / row-only CTAs)
     int n_ccta, r_cls;      // class CTAs per head-instance; retained rows they share (extra CTAs take the rest)
+    float* emit;            // or null: [n_inst][emit_stride][G] every logit (log2 units): the rows, then the class-list entries
+    int emit_stride;
     unsigned long long wait_ns;   // how long a wait on a staging barrier may last (200 ms unless a test shortens it)
     uint32_t tx_extra;      // 0; a test announces more bytes than are copied, so that the cells barrier never completes
     uint32_t zero;          // 0, unknown to the compiler (orders a shared-memory read before a copy into the same bytes)
@@ -568,6 +570,12 @@ decode_staged_kernel(const StagedParams p) {
                 if constexpr (G == 4) { const float4 v = *reinterpret_cast<const float4*>(w + 4 * t); x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w; }
                 else if constexpr (G == 2) { const float2 v = *reinterpret_cast<const float2*>(w + 2 * t); x[0] = v.x; x[1] = v.y; }
                 else x[0] = w[t];
+                if (p.emit) {                                // (same for the whole launch)
+                    float* e = p.emit + ((size_t)u * p.emit_stride + (t < nrows ? rb + t : p.R + cb + (t - nrows))) * G;
+                    if constexpr (G == 4) *reinterpret_cast<float4*>(e) = make_float4(x[0], x[1], x[2], x[3]);
+                    else if constexpr (G == 2) *reinterpret_cast<float2*>(e) = make_float2(x[0], x[1]);
+                    else e[0] = x[0];
+                }
                 float sgn = 1.f;
                 if (t >= nrows) {
                     if (lds_u32(desc_s + (uint32_t)(t - nrows) * 16u + 12u) & (1u << KVR_CL_SIGN_SHIFT)) sgn = -1.f;   // g_0
@@ -843,9 +851,8 @@ bool kvr_decode_staged_plan(const kvr_sketch* sk, int n_inst, int N, int R, int 
 
 cudaError_t kvr_launch_decode_staged(kvr_sketch* sk, int inst0, int n_inst, int N, int R, int rows, const void* q,
                                      const void* Kr, const void* Vr, float scale, float* out,
-                                     const KvrStagedPlan& plan, float* part, uint32_t* tickets, cudaStream_t st) {
-    (void)N;
-    (void)R;
+                                     const KvrStagedPlan& plan, float* part, uint32_t* tickets, float* emit,
+                                     cudaStream_t st) {
     StagedParams p;
     p.q = q;
     p.Kr = (const uint2*)Kr;
@@ -874,6 +881,8 @@ cudaError_t kvr_launch_decode_staged(kvr_sketch* sk, int inst0, int n_inst, int 
     p.zero = 0u;
     p.wait_ns = sk->wait_ns;
     p.tx_extra = sk->tx_extra;
+    p.emit = emit;
+    p.emit_stride = rows + (N - R);
     p.scale_log2e = scale * 1.4426950408889634f;
     sk->launches += 1;
     const bool f16 = sk->d.kv_dtype == KVR_F16;

@@ -64,6 +64,7 @@ struct kvr_sketch {
     int C, logC, n1;     // C = 0: sketch too wide for the staged kernel; n1 = ceil(b / C)
     uint2* clist;        // [n_inst][max_context]  class-ordered entries (format above)
     int32_t* coff;       // [n_inst][C*C+1]        offsets of each class in clist
+    int32_t* ctok;       // [n_inst][max_context]  token index of each clist entry
     int bitmap_words;
 
     // ---- per layer host state ----
@@ -77,6 +78,7 @@ struct kvr_sketch {
     float* ml;                                // [n_inst][G][2] softmax reference maximum (log2 units) and sum of
                                               // the last decode of each head-instance (for score accumulation)
     void* ws_demote; size_t ws_demote_bytes;  // positions / membership of the overflow step
+    void* ws_emit; size_t ws_emit_bytes;      // logits the staged kernel emits for the scored decode call
     void* ws_append; size_t ws_append_bytes;  // storage + new rows before the overflow step of kvr_append
 
     // ---- host-buffer path (allocated on first use) ----
@@ -166,7 +168,13 @@ int kvr_decode_staged_pick_C(int b, int G);
 bool kvr_decode_staged_plan(const kvr_sketch* sk, int n_inst, int N, int R, int rows, bool forced, KvrStagedPlan* plan);
 cudaError_t kvr_launch_decode_staged(kvr_sketch* sk, int inst0, int n_inst, int N, int R, int rows, const void* q,
                                      const void* Kr, const void* Vr, float scale, float* out,
-                                     const KvrStagedPlan& plan, float* part, uint32_t* tickets, cudaStream_t st);
+                                     const KvrStagedPlan& plan, float* part, uint32_t* tickets, float* emit,
+                                     cudaStream_t st);
+// emit (or null): [n_inst][rows + (N - R)][G] logits (log2 units) of the rows, then of the class-list entries;
+// kvr_launch_apply_emitted turns them into attention mass under the launch's final (max, sum) and adds the
+// rows' to score_acc [n_inst][rows], the tokens' to the handle's per-token scores.
+cudaError_t kvr_launch_apply_emitted(kvr_sketch* sk, int inst0, int n_inst, int rows, int a, const float* emit,
+                                     float* score_acc, cudaStream_t st);
 // attention mass of the rows of Kr under the softmax of the layer's last decode, added to acc
 cudaError_t kvr_launch_row_mass(kvr_sketch* sk, int inst0, int n_inst, int rows, const void* q, const void* Kr,
                                 float scale, float* acc, cudaStream_t st);

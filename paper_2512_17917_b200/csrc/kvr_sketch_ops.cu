@@ -38,7 +38,7 @@ insert_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ 
     // Two levels: the rows of one batch (up to INS_UNROLL) are added plainly, in order, and the batch
     // sum goes into a compensated running sum, so the rounding error does not grow with the length
     // of the cell's token list.
-    float s[4] = {0.f, 0.f, 0.f, 0.f}, cc[4] = {0.f, 0.f, 0.f, 0.f}, blk[4];
+    float s[4] = {0.f, 0.f, 0.f, 0.f}, cc[4] = {0.f, 0.f, 0.f, 0.f}, blk[4] = {0.f, 0.f, 0.f, 0.f};
     auto add = [&](uint2 x, uint32_t e) {
         const float2 lo = KvrType<T>::to_f2(x.x), hi = KvrType<T>::to_f2(x.y);
         const float sg = (kv && (e >> 31)) ? -1.f : 1.f;      // g_i(J) for the values, +1 for the keys

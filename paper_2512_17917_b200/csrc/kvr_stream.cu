@@ -82,6 +82,31 @@ vague_mass_kernel(const uint2* __restrict__ q, const float* __restrict__ cells_a
     if (lane == 0) scores_all[(size_t)inst * max_ctx + J] += mass;
 }
 
+// The same two sums from logits a decode kernel already computed (the staged kernel writes them out on
+// request): one thread per logit slot; slot < rows is a retained row, the others are class-list entries,
+// whose token indices the list builder recorded.  No pass over the cache.
+template <int G>
+__global__ void __launch_bounds__(256)
+apply_emitted_kernel(const float* __restrict__ emit, const float* __restrict__ ml_all, const int32_t* __restrict__ ctok_all,
+                     int rows, int a, int max_ctx, int inst0, float* __restrict__ acc, float* __restrict__ scores_all) {
+    const int u = blockIdx.y, inst = inst0 + u;
+    const int slot = blockIdx.x * 256 + threadIdx.x;
+    if (slot >= rows + a) return;
+    const float* e = emit + ((size_t)u * (rows + a) + slot) * G;
+    float x[G];
+    if constexpr (G == 4) { const float4 v = *reinterpret_cast<const float4*>(e); x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w; }
+    else if constexpr (G == 2) { const float2 v = *reinterpret_cast<const float2*>(e); x[0] = v.x; x[1] = v.y; }
+    else x[0] = e[0];
+    float mass = 0.f;
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        const float M = ml_all[((size_t)inst * G + g) * 2], L = ml_all[((size_t)inst * G + g) * 2 + 1];
+        mass += exp2f(x[g] - M) / L;
+    }
+    if (slot < rows) acc[(size_t)u * rows + slot] += mass;
+    else scores_all[(size_t)inst * max_ctx + ctok_all[(size_t)inst * max_ctx + (slot - rows)]] += mass;
+}
+
 __device__ __forceinline__ uint32_t swap_score_key(float s) {      // order-preserving integer image of a float
     const uint32_t u = __float_as_uint(s);
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
@@ -364,6 +389,20 @@ cudaError_t kvr_launch_vague_mass(kvr_sketch* sk, int inst0, int n_inst, int a, 
         default: return cudaErrorInvalidValue;
     }
 #undef KVR_VM
+    sk->launches += 1;
+    return cudaGetLastError();
+}
+
+cudaError_t kvr_launch_apply_emitted(kvr_sketch* sk, int inst0, int n_inst, int rows, int a, const float* emit,
+                                     float* score_acc, cudaStream_t st) {
+    if (rows + a <= 0) return cudaSuccess;
+    const dim3 grid((rows + a + 255) / 256, n_inst);
+    switch (sk->G) {
+        case 1: apply_emitted_kernel<1><<<grid, 256, 0, st>>>(emit, sk->ml, sk->ctok, rows, a, sk->d.max_context, inst0, score_acc, sk->scores); break;
+        case 2: apply_emitted_kernel<2><<<grid, 256, 0, st>>>(emit, sk->ml, sk->ctok, rows, a, sk->d.max_context, inst0, score_acc, sk->scores); break;
+        case 4: apply_emitted_kernel<4><<<grid, 256, 0, st>>>(emit, sk->ml, sk->ctok, rows, a, sk->d.max_context, inst0, score_acc, sk->scores); break;
+        default: return cudaErrorInvalidValue;
+    }
     sk->launches += 1;
     return cudaGetLastError();
 }

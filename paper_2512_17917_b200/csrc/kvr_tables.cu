@@ -110,7 +110,7 @@ __global__ void csr_fill_kernel(const int32_t* __restrict__ tok_h, const int32_t
 // Per head-instance, the token lists the decode kernels walk:
 //   dlist / doff   the compressed tokens (index < N and not retained by the membership bitmap) in
 //                  row-0-cell order, ascending token index inside a cell, as packed entries
-//   clist / coff   (when the handle has a class grid, C > 0) the same tokens regrouped into C x C
+//   clist / coff / ctok  (when the handle has a class grid, C > 0) the same tokens regrouped into C x C
 //                  classes by (row-1 cell mod C, row-2 cell mod C), row-0-cell order kept inside each
 //                  class, the first token of every row-0 cell inside its class flagged and told the
 //                  row-0 cell of the run that follows it
@@ -125,7 +125,8 @@ __global__ void __cluster_dims__(LST_CL, 1, 1) __launch_bounds__(LST_THREADS, 1)
 lists_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ full_list,
              const uint32_t* __restrict__ tok_pack, const uint32_t* __restrict__ bitmap_all, int bitmap_words,
              int b, int N, int max_ctx, int inst0, int n_tbl, int C, int logC, int n1, uint32_t* __restrict__ dlist_all,
-             int32_t* __restrict__ doff_all, uint2* __restrict__ clist_all, int32_t* __restrict__ coff_all) {
+             int32_t* __restrict__ doff_all, uint2* __restrict__ clist_all, int32_t* __restrict__ coff_all,
+             int32_t* __restrict__ ctok_all) {
     extern __shared__ int32_t s_cnt[];        // [cells of this CTA][1 + C * C]: kept tokens, then per class
     __shared__ int32_t s_tot[65];             // column sums over this CTA's cells
     __shared__ int32_t s_all[65];             // column sums over the cluster
@@ -154,12 +155,13 @@ lists_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ f
         return (int)(((h1 & (C - 1)) << logC) | (h2 & (C - 1)));
     };
     // this lane's token of the 32 list positions starting at `base` of a cell that ends at p1
-    auto fetch = [&](int base, int p1, bool& keep, uint32_t& e) {
+    auto fetch = [&](int base, int p1, bool& keep, uint32_t& e, int& J) {
         const int p = base + lane;
         keep = false;
         e = 0u;
+        J = 0;
         if (p < p1) {
-            const int J = full_list[p];
+            J = full_list[p];
             keep = (J < N) && !((bitmap[J >> 5] >> (J & 31)) & 1u);
             if (keep) e = tok_pack[J];
         }
@@ -175,7 +177,8 @@ lists_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ f
         for (int base = p0; base < p1; base += 32) {          // warp-uniform trip count
             bool keep;
             uint32_t e;
-            fetch(base, p1, keep, e);
+            int J;
+            fetch(base, p1, keep, e, J);
             n += __popc(__ballot_sync(0xFFFFFFFFu, keep));
             if (n_cls) {
                 const int k = keep ? cls(e) : 64;
@@ -240,6 +243,7 @@ lists_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ f
     __syncthreads();
     // ---- pass 2: write the lists
     uint2* cl = n_cls ? clist_all + (size_t)inst * max_ctx : nullptr;
+    int32_t* ct = n_cls ? ctok_all + (size_t)inst * max_ctx : nullptr;
     for (int c = c_lo + warp; c < c_hi; c += 32) {
         const int p0 = full_off[c], p1 = full_off[c + 1];
         const int32_t* row = s_cnt + (size_t)(c - c_lo) * n_col;
@@ -251,7 +255,8 @@ lists_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ f
         for (int base = p0; base < p1; base += 32) {
             bool keep;
             uint32_t e;
-            fetch(base, p1, keep, e);
+            int J;
+            fetch(base, p1, keep, e, J);
             const unsigned m = __ballot_sync(0xFFFFFFFFu, keep);
             if (keep) dlist[w + __popc(m & lt)] = e;
             w += __popc(m);
@@ -266,6 +271,7 @@ lists_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ f
                     cl[row[1 + k] + seen] = make_uint2((h1 >> logC) | (((uint32_t)n1 + (h2 >> logC)) << 8),
                                                        ((uint32_t)c << KVR_CL_C0_SHIFT) | (s3 << KVR_CL_SIGN_SHIFT) |
                                                            (seen == 0 ? KVR_CL_FLAG : 0u));
+                    ct[row[1 + k] + seen] = J;
                 }
                 __syncwarp();
                 if (keep && (same & lt) == 0u) s_run[warp][k] += __popc(same);
@@ -347,7 +353,7 @@ cudaError_t kvr_launch_lists(kvr_sketch* sk, int inst0, int n_inst, int N, cudaS
     lists_kernel<<<dim3(LST_CL, n_inst), LST_THREADS, smem, st>>>(sk->full_off, sk->full_list, sk->tok_pack, sk->bitmap,
                                                                   sk->bitmap_words, b, N, sk->d.max_context, inst0, sk->n_tbl, C,
                                                                   sk->logC, sk->n1, sk->dlist, sk->doff, sk->clist,
-                                                                  sk->coff);
+                                                                  sk->coff, sk->ctok);
     sk->launches += 1;
     return cudaGetLastError();
 }

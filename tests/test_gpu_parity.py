@@ -281,6 +281,70 @@ def test_generation_after_compress_scores_and_overflow(which, dtype):
     kvr.kvr_sketch_destroy(sk)
 
 
+@pytest.mark.parametrize("which,dtype,H,Hq,N,b,skew", [("staged", F16, 2, 8, 1800, 40, False), ("staged", BF16, 2, 4, 1800, 9, False),
+                                                       ("staged", F16, 2, 2, 6000, 200, True), ("split", F16, 2, 8, 1800, 40, False),
+                                                       ("split", BF16, 1, 8, 1800, 12, False)])
+def test_scored_decode_keeps_the_scores_of_the_step(which, dtype, H, Hq, N, b, skew):
+    """The decode call that also accumulates the step's attention mass (Calculation Phase: the scores of
+    the step are kept, not computed again): output, row scores and vague-token scores against the oracle,
+    and against the three separate calls on a second handle in the same state.  Two layers in one call
+    (head-instances of the call and of the handle are numbered differently), appended rows, and a hashing
+    that overfills single classes so that the staged kernel takes its tokens in several stretches."""
+    L, B, R, n_new = 2, 1, N // 10, 13
+    G = Hq // H
+    seeds = synth.injective_seeds() if skew else synth.hash_seeds(4242)
+    K, V, Q, q = make_case(4243, B, H, Hq, N + n_new, 8, dtype, L)
+    dev = "cuda"
+    n_inst = L * B * H
+    state = []
+    for _ in range(2):
+        sk = kvr.kvr_sketch_create(b=b, batch=B, n_layers=L, n_kv_heads=H, n_q_heads=Hq, max_context=N + n_new,
+                                   kv_dtype=dtype, hash_seeds=seeds, index_mix=not skew)
+        kvr.kvr_sketch_set_decode_kernel(sk, kvr.KVR_DECODE_SPLIT if which == "split" else kvr.KVR_DECODE_STAGED)
+        Kr, Vr, ret = kvr.kvr_compress(sk, kvr.KVR_ALL_LAYERS, K[..., :N, :].contiguous().to(dev),
+                                       V[..., :N, :].contiguous().to(dev), Q.to(dev), R, 10)
+        state.append((sk, Kr, Vr, ret))
+    sk, Kr, Vr, ret = state[0]
+    cmp0 = kvr.kvr_get_assignment(sk, kvr.KVR_ALL_LAYERS)[0].reshape(n_inst, -1).cpu().numpy()
+    cells_o = orc.insert(inst_major(K)[:, :N], inst_major(V)[:, :N], cmp0, seeds, b, mix=not skew)
+    Kr = torch.cat([Kr, K[..., N:, :].to(dev)], dim=3).contiguous()
+    Vr = torch.cat([Vr, V[..., N:, :].to(dev)], dim=3).contiguous()
+    ret = torch.cat([ret, torch.arange(N, N + n_new, dtype=torch.int32, device=dev).expand(L, B, H, n_new)], dim=3).contiguous()
+    ret_np = ret.reshape(n_inst, -1).cpu().numpy()
+    rows = R + n_new
+    outs, accs, toks = [], [], []
+    for step in range(2):                                   # the second step reuses the workspace of the first
+        qd = synth.make_decode_q(4250 + step, L * B, Hq, 128, dtype, dev).reshape(L, B, Hq, 128)
+        qo = dec_to_inst(qd, H)
+        want = orc.decode(qo, inst_major(Kr), inst_major(Vr), ret_np, cells_o, N + n_new, seeds, mix=not skew)
+        mass = orc.decode_mass(qo, inst_major(Kr), inst_major(Vr), ret_np, cells_o, N + n_new, seeds,
+                               mix=not skew)
+        for k, (h, _, _, _) in enumerate(state):
+            acc = torch.full((L, B, H, rows), 0.25, dtype=torch.float32, device=dev)
+            s0 = kvr.kvr_get_scores(h, kvr.KVR_ALL_LAYERS).reshape(n_inst, -1).cpu().numpy()
+            if k == 0:
+                out = kvr.kvr_decode_attention_scored(h, kvr.KVR_ALL_LAYERS, qd, Kr, Vr, ret, acc)
+            else:
+                out = kvr.kvr_decode_attention(h, kvr.KVR_ALL_LAYERS, qd, Kr, Vr, ret)
+                kvr.kvr_accumulate_scores(h, kvr.KVR_ALL_LAYERS, qd, Kr, acc)
+                kvr.kvr_accumulate_vague_scores(h, kvr.KVR_ALL_LAYERS, qd)
+            assert kvr.kvr_last_decode_kernel(h) == (kvr.KVR_DECODE_SPLIT if which == "split" else kvr.KVR_DECODE_STAGED)
+            assert kvr.kvr_sketch_device_status(h) == 0
+            s1 = kvr.kvr_get_scores(h, kvr.KVR_ALL_LAYERS).reshape(n_inst, -1).cpu().numpy()
+            assert np.abs(out.reshape(n_inst, G, 128).cpu().numpy() - want).max() <= TOL
+            got_rows = acc.reshape(n_inst, rows).cpu().numpy() - 0.25
+            np.testing.assert_allclose(got_rows, np.take_along_axis(mass, ret_np.astype(np.int64), axis=1), rtol=2e-3, atol=2e-6)
+            for u in range(n_inst):
+                np.testing.assert_allclose(s1[u, cmp0[u]] - s0[u, cmp0[u]], mass[u, cmp0[u]], rtol=2e-3, atol=2e-6)
+                assert (s1[u, ret_np[u, :R]] == s0[u, ret_np[u, :R]]).all()        # stored tokens: untouched
+            outs.append(out.clone()); accs.append(got_rows); toks.append(s1 - s0)
+        np.testing.assert_allclose(accs[-2], accs[-1], rtol=2e-4, atol=1e-6)      # one call against the three
+        np.testing.assert_allclose(toks[-2], toks[-1], rtol=2e-4, atol=1e-6)
+        assert torch.equal(outs[-2], outs[-1])
+    for h, _, _, _ in state:
+        kvr.kvr_sketch_destroy(h)
+
+
 @pytest.mark.parametrize("which,dtype,rate", [("staged", F16, 1.1), ("split", BF16, 1.0)])
 def test_swap_loop_and_vague_scores(which, dtype, rate):
     """Algorithm 3's swap loop on the GPU against the oracle: decode, add the attention mass of the
