@@ -34,12 +34,17 @@ kvr_status_t dev_alloc(kvr_sketch* sk, T** p, size_t bytes) {
     return KVR_OK;
 }
 
-// Grow a workspace; cudaFree orders itself after all work already enqueued on the device.
+// Grow a workspace; cudaFree orders itself after all work already enqueued on the device.  A workspace
+// that has to grow again gets a quarter more than asked for: a generation loop, whose storage grows by
+// a row per step, then reallocates (and synchronises the device) once in many steps, not in every one.
 kvr_status_t ensure(kvr_sketch* sk, void** p, size_t* cur, size_t need) {
     if (need <= *cur) return KVR_OK;
+    const size_t want = *p ? need + need / 4 : need;
     if (*p) { cudaFree(*p); sk->device_bytes -= *cur; *p = nullptr; *cur = 0; }
     need = (need + 255) & ~(size_t)255;
-    cudaError_t e = cudaMalloc(p, need);
+    cudaError_t e = cudaMalloc(p, (want + 255) & ~(size_t)255);
+    if (e == cudaSuccess) need = (want + 255) & ~(size_t)255;
+    else { cudaGetLastError(); e = cudaMalloc(p, need); }       // no room for the headroom: the exact size
     if (e != cudaSuccess) { cudaGetLastError(); *p = nullptr; return KVR_ERR_ALLOC; }
     *cur = need;
     sk->device_bytes += need;

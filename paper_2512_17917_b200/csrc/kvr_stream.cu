@@ -131,97 +131,348 @@ __device__ __forceinline__ unsigned long long swap_block_reduce(unsigned long lo
     return r;                                                     // the same value in every thread
 }
 
-// The swap loop of Algorithm 3, one CTA per head-instance (the loop is sequential by construction).
+// ---- the swap loop of Algorithm 3, one CTA of 1024 threads per head-instance ------------------------
 // Candidate part = rows [0, rows - n_recent); Vague part = the `a` tokens listed in cmp (their scores
 // in the handle's per-token array).  Equal scores: the lower token index is taken, for the minimum
 // and for the maximum.  The decision C.Min * ReplaceRate < V.Max is taken in fp32.
+struct SwapArgs {
+    int32_t* ret; float* rs; float* scores; int32_t* cmp; uint32_t* bitmap; float* cK; float* cV;
+    const int32_t* tok_h; const int8_t* tok_g;
+    int n_cand, a, max_ctx, b, mean;
+    float rate;
+};
+__device__ __forceinline__ unsigned long long swap_cand_key(const SwapArgs& A, int r) {      // smallest = worst candidate
+    return ((unsigned long long)swap_score_key(A.rs[r]) << 32) | (uint32_t)A.ret[r];
+}
+__device__ __forceinline__ unsigned long long swap_vague_key(const SwapArgs& A, int t) {     // smallest = best vague token
+    const int J = A.cmp[t];
+    return ((unsigned long long)(~swap_score_key(A.scores[J])) << 32) | (uint32_t)J;
+}
+
+// One swap, by threads 0..255 (keys | values x channel) and one bookkeeping thread; the caller
+// synchronises before (the pair is read by everybody) and after.
+template <typename T>
+__device__ __forceinline__ void swap_one(const SwapArgs& A, T* Kr, T* Vr, int row, int pos, int tid) {
+    const int Jc = A.ret[row], Jv = A.cmp[pos];
+    const float c_min = A.rs[row], v_max = A.scores[Jv];
+    __syncthreads();                                          // everybody has read the pair before it is rewritten
+    if (tid < 2 * KVR_D) {
+        const int d = tid & (KVR_D - 1);
+        const bool val = tid >= KVR_D;
+        float* cells = val ? A.cV : A.cK;
+        T* rowp = (val ? Vr : Kr) + (size_t)row * KVR_D + d;
+        float x[KVR_R], g[KVR_R];
+        size_t cell[KVR_R];
+#pragma unroll
+        for (int i = 0; i < KVR_R; ++i) {
+            cell[i] = ((size_t)i * A.b + A.tok_h[(size_t)i * A.max_ctx + Jv]) * KVR_D + d;
+            g[i] = val ? (float)A.tok_g[(size_t)i * A.max_ctx + Jv] : 1.f;
+            x[i] = g[i] * cells[cell[i]];
+        }
+        const float m = kvr_comb3(x[0], x[1], x[2], A.mean);        // query the vague token (Algorithm 2)
+#pragma unroll
+        for (int i = 0; i < KVR_R; ++i) cells[cell[i]] -= g[i] * m; // take it out of the sketch again
+        const float c = KvrType<T>::to_float(*rowp);
+#pragma unroll
+        for (int i = 0; i < KVR_R; ++i) {                           // the candidate's vectors go in (Algorithm 1)
+            const size_t cc = ((size_t)i * A.b + A.tok_h[(size_t)i * A.max_ctx + Jc]) * KVR_D + d;
+            cells[cc] += (val ? (float)A.tok_g[(size_t)i * A.max_ctx + Jc] : 1.f) * c;
+        }
+        *rowp = KvrType<T>::from_float(m);                          // the queried vectors take its row
+    }
+    if (tid == 1023) {
+        A.ret[row] = Jv;
+        A.rs[row] = v_max;
+        A.scores[Jc] = c_min;
+        A.cmp[pos] = Jc;
+        atomicOr(&A.bitmap[Jv >> 5], 1u << (Jv & 31));
+        atomicAnd(&A.bitmap[Jc >> 5], ~(1u << (Jc & 31)));
+    }
+}
+
+// The loop as the algorithm prints it: find the pair, decide, swap, again.
+template <typename T>
+__device__ int swap_loop_in_order(const SwapArgs& A, T* Kr, T* Vr, int done, int max_swaps, unsigned long long* s_w, int* s_pair) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (; done < max_swaps; ++done) {
+        unsigned long long best = ~0ull;
+        int best_i = -1;
+        for (int r = tid; r < A.n_cand; r += 1024) {
+            const unsigned long long key = swap_cand_key(A, r);
+            if (key < best) { best = key; best_i = r; }
+        }
+        const unsigned long long cmin = swap_block_reduce<false>(best, s_w, lane, warp);
+        if (best_i >= 0 && best == cmin) s_pair[0] = best_i;
+        best = ~0ull;
+        best_i = -1;
+        for (int t = tid; t < A.a; t += 1024) {
+            const unsigned long long key = swap_vague_key(A, t);
+            if (key < best) { best = key; best_i = t; }
+        }
+        const unsigned long long vmax = swap_block_reduce<false>(best, s_w, lane, warp);
+        if (best_i >= 0 && best == vmax) s_pair[1] = best_i;
+        __syncthreads();
+        const int row = s_pair[0], pos = s_pair[1];
+        if (!(__fmul_rn(A.rs[row], A.rate) < A.scores[A.cmp[pos]])) break;      // (uniform)
+        swap_one<T>(A, Kr, Vr, row, pos, tid);
+        __syncthreads();                                          // the next round sees this one's writes
+    }
+    return done;
+}
+
+// The K smallest of n distinct 64-bit keys (hi(i) << 32 | lo(i)), ascending: their positions go to
+// out_pos[0..K).  All 1024 threads call it.  hi(i) is cheap (the caller keeps the score images in
+// shared memory where they fit); lo(i) reads global memory.
+//   1. Every thread takes the smallest high word of its own keys (i = tid, tid + 1024, ...); the
+//      K-th smallest of these 1024 minima, U, bounds the K-th key from above, because K different
+//      keys lie at or below it.
+//   2. The keys with high word <= U are collected (normally a small multiple of K) and sorted.
+//   3. Should they not fit (more than SW_M: many equal scores), the K-th key is found bit by bit
+//      instead: T grows from the top bit down while fewer than K keys lie below it, one count over
+//      all keys per bit; then the same among the low words of the keys that share T.
+constexpr int SW_K = 256, SW_M = 2048;
+__device__ __forceinline__ int swap_block_sum(int v, int* s_cnt) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    if (lane == 0) s_cnt[warp] = v;
+    __syncthreads();
+    int t = s_cnt[lane];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
+    __syncthreads();
+    return t;                                                     // the same value in every thread
+}
+template <class HiFn, class LoFn>
+__device__ void swap_select(int n, int K, HiFn hi, LoFn lo, unsigned long long* s_lk, int* s_lp, int* s_cnt, int* s_misc,
+                            int* out_pos) {
+    const int tid = threadIdx.x, lane = tid & 31;
+    // ---- 1. the K-th smallest of the threads' minima
+    uint32_t U;
+    {
+        uint32_t mn = 0xFFFFFFFFu;
+        for (int i = tid; i < n; i += 1024) mn = min(mn, hi(i));
+        if (tid == 0) s_misc[2] = 0;
+        // U = the largest value with fewer than K minima below it, bit by bit (one barrier per bit)
+        U = 0u;
+        for (int bit = 31; bit >= 0; --bit) {
+            const uint32_t trial = U | (1u << bit);
+            if (__syncthreads_count(mn < trial) < K) U = trial;
+        }
+    }
+    // ---- 2. the keys at or below U (a warp reserves its places with one addition)
+    for (int base = 0; base < n; base += 1024) {
+        const int i = base + tid;
+        uint32_t h = 0u;
+        const bool in = i < n && (h = hi(i)) <= U;
+        const unsigned m = __ballot_sync(0xFFFFFFFFu, in);
+        int at = 0;
+        if (lane == 0 && m) at = atomicAdd(&s_misc[2], __popc(m));
+        at = __shfl_sync(0xFFFFFFFFu, at, 0) + __popc(m & ((1u << lane) - 1u));
+        if (in && at < SW_M) {
+            s_lk[at] = ((unsigned long long)h << 32) | lo(i);
+            s_lp[at] = i;
+        }
+    }
+    __syncthreads();
+    int M = s_misc[2];
+    __syncthreads();
+    if (M > SW_M) {
+        // ---- 3. too many: find the K-th key bit by bit and collect up to it
+        uint32_t T = 0u;
+        int less = 0;                                             // keys whose high word is below T
+        for (int bit = 31; bit >= 0; --bit) {
+            const uint32_t trial = T | (1u << bit);
+            int c = 0;
+            for (int i = tid; i < n; i += 1024) c += hi(i) < trial ? 1 : 0;
+            c = swap_block_sum(c, s_cnt);
+            if (c < K) { T = trial; less = c; }
+        }
+        int ties = 0;
+        for (int i = tid; i < n; i += 1024) ties += hi(i) == T ? 1 : 0;
+        ties = swap_block_sum(ties, s_cnt);
+        uint32_t TL = 0xFFFFFFFFu;
+        const int need = K - less;                                // of the `ties` keys with high word T
+        if (ties > need) {
+            TL = 0u;
+            for (int bit = 31; bit >= 0; --bit) {
+                const uint32_t trial = TL | (1u << bit);
+                int c = 0;
+                for (int i = tid; i < n; i += 1024)
+                    if (hi(i) == T) c += lo(i) < trial ? 1 : 0;
+                c = swap_block_sum(c, s_cnt);
+                if (c < need) TL = trial;
+            }
+        }
+        if (tid == 0) s_misc[2] = 0;
+        __syncthreads();
+        for (int i = tid; i < n; i += 1024) {
+            const uint32_t h = hi(i);
+            if (h <= T) {
+                const uint32_t l = lo(i);
+                if (h < T || l <= TL) {
+                    const int at = atomicAdd(&s_misc[2], 1);
+                    if (at < SW_M) {                              // (keys that are not distinct would give more than K)
+                        s_lk[at] = ((unsigned long long)h << 32) | l;
+                        s_lp[at] = i;
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        M = min(s_misc[2], SW_M);
+        __syncthreads();
+    }
+    int P = 2;
+    while (P < M) P <<= 1;
+    for (int i = M + tid; i < P; i += 1024) { s_lk[i] = ~0ull; s_lp[i] = 0; }
+    __syncthreads();
+    for (int k = 2; k <= P; k <<= 1)
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int i = tid; i < P; i += 1024) {
+                const int x = i ^ j;
+                if (x > i) {
+                    const unsigned long long ka = s_lk[i], kb = s_lk[x];
+                    if ((ka > kb) == ((i & k) == 0)) {
+                        s_lk[i] = kb; s_lk[x] = ka;
+                        const int pa = s_lp[i]; s_lp[i] = s_lp[x]; s_lp[x] = pa;
+                    }
+                }
+            }
+            __syncthreads();
+        }
+    if (tid < K) out_pos[tid] = s_lp[tid];
+    __syncthreads();
+}
+
+// With ReplaceRate >= 1 and scores >= 0 the loop never touches a token twice: a token that has just
+// become a candidate scores more than the minimum it replaced times the rate, so once it is the
+// minimum the test fails; a token that has just become vague scores less than the maximum it
+// replaced, so once it is the maximum the test fails as well.  The k-th swap therefore pairs the
+// k-th worst candidate with the k-th best vague token of the lists as they stand at entry, up to
+// the first pair that fails the test: both lists are selected and sorted in parallel (up to SW_K
+// pairs per round), and only the updates of the cells, which do depend on their order, run one
+// after the other, without any search in between.  Other rates or scores take the loop in order.
 template <typename T>
 __global__ void __launch_bounds__(1024)
 swap_kernel(T* __restrict__ Kr_all, T* __restrict__ Vr_all, int32_t* __restrict__ ret_all, float* __restrict__ rs_all,
             int rows, int n_recent, float rate, int max_swaps, float* __restrict__ scores_all,
             int32_t* __restrict__ cmp_all, int a, uint32_t* __restrict__ bitmap_all, int bitmap_words,
             float* __restrict__ cells_all, const int32_t* __restrict__ tok_h, const int8_t* __restrict__ tok_g,
-            int max_ctx, int b, int inst0, int n_tbl, int mean, int32_t* __restrict__ n_swapped) {
+            int max_ctx, int b, int inst0, int n_tbl, int mean, int n_cache, int32_t* __restrict__ n_swapped) {
+    extern __shared__ uint32_t s_img[];                          // score images of the first n_cache candidates, then vague tokens
     __shared__ unsigned long long s_w[32];
-    __shared__ int s_row, s_pos;
-    const int u = blockIdx.x, inst = inst0 + u, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    tok_h += (size_t)(n_tbl > 1 ? inst % n_tbl : 0) * KVR_R * max_ctx;
-    tok_g += (size_t)(n_tbl > 1 ? inst % n_tbl : 0) * KVR_R * max_ctx;
+    __shared__ unsigned long long s_lk[SW_M];                    // scratch of the selection: keys, positions
+    __shared__ int s_lp[SW_M];
+    __shared__ int s_posC[SW_K], s_posV[SW_K], s_Jc[SW_K], s_Jv[SW_K];
+    __shared__ float s_c[SW_K], s_v[SW_K];
+    __shared__ uint16_t s_hC[SW_K][KVR_R], s_hV[SW_K][KVR_R];     // cell index | sign bit << 15
+    __shared__ int s_cnt[32], s_misc[4], s_pair[2], s_nsw;
+    const int u = blockIdx.x, inst = inst0 + u, tid = threadIdx.x;
+    SwapArgs A;
+    A.tok_h = tok_h + (size_t)(n_tbl > 1 ? inst % n_tbl : 0) * KVR_R * max_ctx;
+    A.tok_g = tok_g + (size_t)(n_tbl > 1 ? inst % n_tbl : 0) * KVR_R * max_ctx;
     T* Kr = Kr_all + (size_t)u * rows * KVR_D;
     T* Vr = Vr_all + (size_t)u * rows * KVR_D;
-    int32_t* ret = ret_all + (size_t)u * rows;
-    float* rs = rs_all + (size_t)u * rows;
-    float* scores = scores_all + (size_t)inst * max_ctx;
-    int32_t* cmp = cmp_all + (size_t)inst * max_ctx;
-    uint32_t* bitmap = bitmap_all + (size_t)inst * bitmap_words;
-    float* cK = cells_all + (size_t)inst * 2 * KVR_R * b * KVR_D;
-    float* cV = cK + (size_t)KVR_R * b * KVR_D;
-    const int n_cand = rows - n_recent;
+    A.ret = ret_all + (size_t)u * rows;
+    A.rs = rs_all + (size_t)u * rows;
+    A.scores = scores_all + (size_t)inst * max_ctx;
+    A.cmp = cmp_all + (size_t)inst * max_ctx;
+    A.bitmap = bitmap_all + (size_t)inst * bitmap_words;
+    A.cK = cells_all + (size_t)inst * 2 * KVR_R * b * KVR_D;
+    A.cV = A.cK + (size_t)KVR_R * b * KVR_D;
+    A.n_cand = rows - n_recent;
+    A.a = a; A.max_ctx = max_ctx; A.b = b; A.mean = mean; A.rate = rate;
     int done = 0;
-    if (n_cand > 0 && a > 0) {
-        for (; done < max_swaps; ++done) {
-            // worst candidate: lowest (score, token index)
-            unsigned long long best = ~0ull;
-            int best_i = -1;
-            for (int r = tid; r < n_cand; r += 1024) {
-                const unsigned long long key = ((unsigned long long)swap_score_key(rs[r]) << 32) | (uint32_t)ret[r];
-                if (key < best) { best = key; best_i = r; }
-            }
-            const unsigned long long cmin = swap_block_reduce<false>(best, s_w, lane, warp);
-            if (best_i >= 0 && best == cmin) s_row = best_i;
-            // best vague token: highest score, then lowest token index
-            best = 0ull;
-            best_i = -1;
-            for (int t = tid; t < a; t += 1024) {
-                const int J = cmp[t];
-                const unsigned long long key = ((unsigned long long)swap_score_key(scores[J]) << 32) | (0xFFFFFFFFu - (uint32_t)J);
-                if (key > best) { best = key; best_i = t; }
-            }
-            const unsigned long long vmax = swap_block_reduce<true>(best, s_w, lane, warp);
-            if (best_i >= 0 && best == vmax) s_pos = best_i;
-            __syncthreads();
-            const int row = s_row, pos = s_pos;
-            const int Jc = ret[row], Jv = cmp[pos];
-            const float c_min = rs[row], v_max = scores[Jv];
-            if (!(__fmul_rn(c_min, rate) < v_max)) break;         // (uniform)
-            __syncthreads();                                      // everybody has read the pair before it is rewritten
-            if (tid < KVR_D) {
-                const int d = tid;
-                float kk[KVR_R], vv[KVR_R], gv[KVR_R];
-                size_t cell[KVR_R];
+    if (A.n_cand > 0 && a > 0 && max_swaps > 0) {
+        // a score with its sign bit set, or a rate below one: the argument above does not hold
+        int odd = !(rate >= 1.f);
+        const int nc_c = min(A.n_cand, n_cache), nc_v = min(a, n_cache - nc_c);
+        for (int r = tid; r < A.n_cand; r += 1024) {
+            const float sc = A.rs[r];
+            odd |= (int)(__float_as_uint(sc) >> 31);
+            if (r < nc_c) s_img[r] = swap_score_key(sc);
+        }
+        for (int t = tid; t < a; t += 1024) {
+            const float sc = A.scores[A.cmp[t]];
+            odd |= (int)(__float_as_uint(sc) >> 31);
+            if (t < nc_v) s_img[nc_c + t] = ~swap_score_key(sc);
+        }
+        odd = __syncthreads_or(odd);
+        if (odd) {
+            done = swap_loop_in_order<T>(A, Kr, Vr, 0, max_swaps, s_w, s_pair);
+        } else {
+            for (;;) {
+                const int K = min(min(max_swaps - done, SW_K), min(A.n_cand, a));
+                swap_select(A.n_cand, K, [&](int r) { return r < nc_c ? s_img[r] : swap_score_key(A.rs[r]); },
+                            [&](int r) { return (uint32_t)A.ret[r]; }, s_lk, s_lp, s_cnt, s_misc, s_posC);
+                swap_select(a, K, [&](int t) { return t < nc_v ? s_img[nc_c + t] : ~swap_score_key(A.scores[A.cmp[t]]); },
+                            [&](int t) { return (uint32_t)A.cmp[t]; }, s_lk, s_lp, s_cnt, s_misc, s_posV);
+                if (tid == 0) s_nsw = K;
+                __syncthreads();
+                if (tid < K) {
+                    const int row = s_posC[tid], pos = s_posV[tid];
+                    const int Jc = A.ret[row], Jv = A.cmp[pos];
+                    const float c = A.rs[row], v = A.scores[Jv];
+                    s_Jc[tid] = Jc; s_Jv[tid] = Jv; s_c[tid] = c; s_v[tid] = v;
 #pragma unroll
-                for (int i = 0; i < KVR_R; ++i) {
-                    cell[i] = ((size_t)i * b + tok_h[(size_t)i * max_ctx + Jv]) * KVR_D + d;
-                    gv[i] = (float)tok_g[(size_t)i * max_ctx + Jv];
-                    kk[i] = cK[cell[i]];
-                    vv[i] = gv[i] * cV[cell[i]];
+                    for (int i = 0; i < KVR_R; ++i) {
+                        s_hC[tid][i] = (uint16_t)(A.tok_h[(size_t)i * max_ctx + Jc] | (A.tok_g[(size_t)i * max_ctx + Jc] < 0 ? 0x8000 : 0));
+                        s_hV[tid][i] = (uint16_t)(A.tok_h[(size_t)i * max_ctx + Jv] | (A.tok_g[(size_t)i * max_ctx + Jv] < 0 ? 0x8000 : 0));
+                    }
+                    if (!(__fmul_rn(c, rate) < v)) atomicMin(&s_nsw, tid);          // the loop ends at the first such pair
                 }
-                const float Kt = kvr_comb3(kk[0], kk[1], kk[2], mean), Vt = kvr_comb3(vv[0], vv[1], vv[2], mean);   // query the vague token (Algorithm 2)
+                __syncthreads();
+                const int n_sw = s_nsw;
+                if (tid < 2 * KVR_D) {                            // the cells and the rows, swap after swap
+                    const int d = tid & (KVR_D - 1);
+                    const bool val = tid >= KVR_D;
+                    float* cells = (val ? A.cV : A.cK) + d;
+                    T* rowsp = (val ? Vr : Kr) + d;
+                    for (int k = 0; k < n_sw; ++k) {
+                        // everything the swap reads is asked for at once (one round trip to memory per swap);
+                        // where the candidate's cell is the vague token's own, it takes the value just computed
+                        float xv[KVR_R], xc[KVR_R], gv[KVR_R], gc[KVR_R];
+                        size_t cv[KVR_R], cc[KVR_R];
+                        T* rp = rowsp + (size_t)s_posC[k] * KVR_D;
 #pragma unroll
-                for (int i = 0; i < KVR_R; ++i) {                 // take it out of the sketch again
-                    cK[cell[i]] -= Kt;
-                    cV[cell[i]] -= gv[i] * Vt;
-                }
-                const float kc = KvrType<T>::to_float(Kr[(size_t)row * KVR_D + d]);
-                const float vc = KvrType<T>::to_float(Vr[(size_t)row * KVR_D + d]);
+                        for (int i = 0; i < KVR_R; ++i) {
+                            const uint32_t ev = s_hV[k][i], ec = s_hC[k][i];
+                            cv[i] = ((size_t)i * b + (ev & 0x7FFFu)) * KVR_D;
+                            cc[i] = ((size_t)i * b + (ec & 0x7FFFu)) * KVR_D;
+                            gv[i] = (val && (ev & 0x8000u)) ? -1.f : 1.f;
+                            gc[i] = (val && (ec & 0x8000u)) ? -1.f : 1.f;
+                            xv[i] = cells[cv[i]];
+                            xc[i] = cells[cc[i]];
+                        }
+                        const float c = KvrType<T>::to_float(*rp);
+                        const float m = kvr_comb3(gv[0] * xv[0], gv[1] * xv[1], gv[2] * xv[2], mean);    // Algorithm 2
 #pragma unroll
-                for (int i = 0; i < KVR_R; ++i) {                 // the candidate's vectors go in (Algorithm 1)
-                    const size_t cc = ((size_t)i * b + tok_h[(size_t)i * max_ctx + Jc]) * KVR_D + d;
-                    cK[cc] += kc;
-                    cV[cc] += (float)tok_g[(size_t)i * max_ctx + Jc] * vc;
+                        for (int i = 0; i < KVR_R; ++i) {
+                            const float nv = xv[i] - gv[i] * m;               // the vague token leaves the sketch
+                            const float nc = (cc[i] == cv[i] ? nv : xc[i]) + gc[i] * c;              // the candidate enters it (Algorithm 1)
+                            cells[cv[i]] = nv;
+                            cells[cc[i]] = nc;
+                        }
+                        *rp = KvrType<T>::from_float(m);
+                    }
+                } else {                                          // who is where, and with which score
+                    for (int k = tid - 2 * KVR_D; k < n_sw; k += 1024 - 2 * KVR_D) {
+                        const int row = s_posC[k], pos = s_posV[k], Jc = s_Jc[k], Jv = s_Jv[k];
+                        A.ret[row] = Jv;
+                        A.rs[row] = s_v[k];
+                        A.scores[Jc] = s_c[k];
+                        A.cmp[pos] = Jc;
+                        if (row < nc_c) s_img[row] = swap_score_key(s_v[k]);
+                        if (pos < nc_v) s_img[nc_c + pos] = ~swap_score_key(s_c[k]);
+                        atomicOr(&A.bitmap[Jv >> 5], 1u << (Jv & 31));
+                        atomicAnd(&A.bitmap[Jc >> 5], ~(1u << (Jc & 31)));
+                    }
                 }
-                Kr[(size_t)row * KVR_D + d] = KvrType<T>::from_float(Kt);                            // the queried vectors take its row
-                Vr[(size_t)row * KVR_D + d] = KvrType<T>::from_float(Vt);
+                done += n_sw;
+                __syncthreads();
+                if (n_sw < K || K < SW_K || done >= max_swaps) break;
             }
-            if (tid == 1023) {
-                ret[row] = Jv;
-                rs[row] = v_max;
-                scores[Jc] = c_min;
-                cmp[pos] = Jc;
-                atomicOr(&bitmap[Jv >> 5], 1u << (Jv & 31));
-                atomicAnd(&bitmap[Jc >> 5], ~(1u << (Jc & 31)));
-            }
-            __syncthreads();                                      // the next round sees this one's writes
         }
     }
     if (tid == 0 && n_swapped) n_swapped[u] = done;
@@ -291,7 +542,8 @@ insert_rows_kernel(const int32_t* __restrict__ tok_h, const int8_t* __restrict__
     *cell = v;
 }
 
-// Ascending list of the compressed tokens (index < N, membership bit clear) of one head-instance.
+// Ascending list of the compressed tokens (index < N, membership bit clear) of one head-instance:
+// a thread takes 32 tokens (one bitmap word) at a time, the CTA scans the counts.
 __global__ void __launch_bounds__(1024)
 cmp_from_bitmap_kernel(const uint32_t* __restrict__ bitmap_all, int bitmap_words, int N, int max_ctx, int inst0,
                        int32_t* __restrict__ cmp_all) {
@@ -300,19 +552,41 @@ cmp_from_bitmap_kernel(const uint32_t* __restrict__ bitmap_all, int bitmap_words
     const int inst = inst0 + blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t* bitmap = bitmap_all + (size_t)inst * bitmap_words;
     int32_t* cmp = cmp_all + (size_t)inst * max_ctx;
+    const int words = (N + 31) >> 5;
     if (tid == 0) s_run = 0;
     __syncthreads();
-    for (int base = 0; base < N; base += 1024) {
-        const int J = base + tid;
-        const bool out = (J < N) && !((bitmap[J >> 5] >> (J & 31)) & 1u);
-        const unsigned m = __ballot_sync(0xFFFFFFFFu, out);
-        if (lane == 0) s_warp[warp] = __popc(m);
+    for (int base = 0; base < words; base += 1024) {
+        const int w = base + tid;
+        uint32_t out = 0u;                                        // bit set = compressed token
+        if (w < words) {
+            out = ~bitmap[w];
+            if (w == words - 1 && (N & 31)) out &= (1u << (N & 31)) - 1u;
+        }
+        const int n = __popc(out);
+        int inc = n;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+            if (lane >= o) inc += t;
+        }
+        if (lane == 31) s_warp[warp] = inc;
         __syncthreads();
-        int before = s_run + __popc(m & ((1u << lane) - 1u));
-        for (int w = 0; w < warp; ++w) before += s_warp[w];
-        if (out) cmp[before] = J;
+        int wsum = s_warp[lane], winc = wsum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, winc, o);
+            if (lane >= o) winc += t;
+        }
+        const int before_warp = __shfl_sync(0xFFFFFFFFu, winc - wsum, warp);
+        const int total = __shfl_sync(0xFFFFFFFFu, winc, 31);
+        const int at = s_run + before_warp + inc - n;
+        for (int l = 0; l < 32; ++l) {                            // word by word: a warp writes neighbouring entries
+            const uint32_t m = __shfl_sync(0xFFFFFFFFu, out, l);
+            const int at_l = __shfl_sync(0xFFFFFFFFu, at, l);
+            if ((m >> lane) & 1u) cmp[at_l + __popc(m & ((1u << lane) - 1u))] = ((base + (warp << 5) + l) << 5) + lane;
+        }
         __syncthreads();
-        if (tid == 1023) s_run = before + (out ? 1 : 0);
+        if (tid == 0) s_run += total;
         __syncthreads();
     }
 }
@@ -412,15 +686,26 @@ cudaError_t kvr_launch_swap(kvr_sketch* sk, int inst0, int n_inst, int N, int a,
                             float* row_scores, int rows, int n_recent, float rate, int max_swaps, int32_t* n_swapped,
                             cudaStream_t st) {
     const int mc = sk->d.max_context;
-    if (sk->d.kv_dtype == KVR_F16)
-        swap_kernel<__half><<<n_inst, 1024, 0, st>>>((__half*)Kr, (__half*)Vr, ret_idx, row_scores, rows, n_recent, rate,
-                                                     max_swaps, sk->scores, sk->cmp_idx, a, sk->bitmap, sk->bitmap_words,
-                                                     sk->cells, sk->tok_h, sk->tok_g, mc, sk->d.b, inst0, sk->n_tbl, sk->combine, n_swapped);
-    else
-        swap_kernel<__nv_bfloat16><<<n_inst, 1024, 0, st>>>((__nv_bfloat16*)Kr, (__nv_bfloat16*)Vr, ret_idx, row_scores,
-                                                            rows, n_recent, rate, max_swaps, sk->scores, sk->cmp_idx, a,
-                                                            sk->bitmap, sk->bitmap_words, sk->cells, sk->tok_h,
-                                                            sk->tok_g, mc, sk->d.b, inst0, sk->n_tbl, sk->combine, n_swapped);
+    // shared memory for the score images of candidates and vague tokens, as many as fit
+    const int n_cache = std::min(std::max(rows - n_recent, 0) + a, (int)((160 * 1024) / sizeof(uint32_t)));
+    const size_t smem = sizeof(uint32_t) * (size_t)std::max(n_cache, 1);
+    cudaError_t e0 = cudaSuccess;
+    if (sk->d.kv_dtype == KVR_F16) {
+        e0 = cudaFuncSetAttribute(swap_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e0 != cudaSuccess) return e0;
+        swap_kernel<__half><<<n_inst, 1024, smem, st>>>((__half*)Kr, (__half*)Vr, ret_idx, row_scores, rows, n_recent, rate,
+                                                        max_swaps, sk->scores, sk->cmp_idx, a, sk->bitmap, sk->bitmap_words,
+                                                        sk->cells, sk->tok_h, sk->tok_g, mc, sk->d.b, inst0, sk->n_tbl,
+                                                        sk->combine, n_cache, n_swapped);
+    } else {
+        e0 = cudaFuncSetAttribute(swap_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e0 != cudaSuccess) return e0;
+        swap_kernel<__nv_bfloat16><<<n_inst, 1024, smem, st>>>((__nv_bfloat16*)Kr, (__nv_bfloat16*)Vr, ret_idx, row_scores,
+                                                               rows, n_recent, rate, max_swaps, sk->scores, sk->cmp_idx, a,
+                                                               sk->bitmap, sk->bitmap_words, sk->cells, sk->tok_h,
+                                                               sk->tok_g, mc, sk->d.b, inst0, sk->n_tbl, sk->combine,
+                                                               n_cache, n_swapped);
+    }
     cmp_from_bitmap_kernel<<<n_inst, 1024, 0, st>>>(sk->bitmap, sk->bitmap_words, N, mc, inst0, sk->cmp_idx);
     sk->launches += 2;
     cudaError_t e = cudaGetLastError();

@@ -345,7 +345,7 @@ def test_scored_decode_keeps_the_scores_of_the_step(which, dtype, H, Hq, N, b, s
         kvr.kvr_sketch_destroy(h)
 
 
-@pytest.mark.parametrize("which,dtype,rate", [("staged", F16, 1.1), ("split", BF16, 1.0)])
+@pytest.mark.parametrize("which,dtype,rate", [("staged", F16, 1.1), ("split", BF16, 1.0), ("staged", F16, 0.9)])
 def test_swap_loop_and_vague_scores(which, dtype, rate):
     """Algorithm 3's swap loop on the GPU against the oracle: decode, add the attention mass of the
     vague tokens to the per-token scores and of the stored rows to the row scores, then swap.  Which
@@ -405,13 +405,46 @@ def test_swap_loop_and_vague_scores(which, dtype, rate):
         assert np.abs(cells_g[u] - co).max() <= TOL
         dk, dv = np.abs(inst_major(Kr)[u] - Ko), np.abs(inst_major(Vr)[u] - Vo)
         assert (dk <= TOL + 2 * ulp * np.abs(Ko)).all() and (dv <= TOL + 2 * ulp * np.abs(Vo)).all()
-        untouched = ro == ret_np[u]
-        assert (inst_major(Kr)[u][untouched] == Kr_b[u][untouched]).all()
+        if rate >= 1.0:                      # (below one a token can leave and come back: its row is then a queried one)
+            untouched = ro == ret_np[u]
+            assert (inst_major(Kr)[u][untouched] == Kr_b[u][untouched]).all()
         new_cells.append(co)
     # ---- the lists were rebuilt: the next decode sees the swapped storage
     out = kvr.kvr_decode_attention(sk, 0, qd, Kr, Vr, ret)
     want = orc.decode(qo, inst_major(Kr), inst_major(Vr), ret_g, np.stack(new_cells), N, seeds)
     assert np.abs(out.reshape(n_inst, G, 128).cpu().numpy() - want).max() <= TOL
+    kvr.kvr_sketch_destroy(sk)
+
+
+def test_swap_loop_with_equal_candidate_scores():
+    """Thousands of candidates with the same score: which of them the swap loop gives up is decided by
+    the token index alone (the lowest first), and the selection cannot keep all the ties in its
+    scratch.  Row indices, row scores and the number of swaps against the oracle, exactly."""
+    B, H, Hq, N, R, b, n_rec, limit = 1, 2, 2, 6000, 3200, 60, 8, 40
+    seeds = synth.hash_seeds(717)
+    K, V, Q, q = make_case(718, B, H, Hq, N, 8, F16, 1)
+    dev = "cuda"
+    sk = kvr.kvr_sketch_create(b=b, batch=B, n_layers=1, n_kv_heads=H, n_q_heads=Hq, max_context=N, kv_dtype=F16,
+                               hash_seeds=seeds)
+    Kr, Vr, ret = kvr.kvr_compress(sk, 0, K[0].to(dev), V[0].to(dev), Q[0].to(dev), R, n_rec)
+    n_inst = B * H
+    ret_np = ret.reshape(n_inst, -1).cpu().numpy().copy()
+    cmp0 = kvr.kvr_get_assignment(sk, 0)[0].reshape(n_inst, -1).cpu().numpy()
+    cells_o = orc.insert(inst_major(K[0]), inst_major(V[0]), cmp0, seeds, b)
+    s1 = kvr.kvr_get_scores(sk, 0).reshape(n_inst, N).cpu().numpy()
+    acc = torch.full((B, H, R), 1e-12, dtype=torch.float32, device=dev)          # every candidate the same, below every vague token
+    acc_np = acc.reshape(n_inst, -1).cpu().numpy().copy()
+    Kr_b, Vr_b = inst_major(Kr).copy(), inst_major(Vr).copy()
+    rounder = lambda x: torch.from_numpy(np.asarray(x, np.float64)).to(F16).double().numpy()
+    n_sw = kvr.kvr_swap(sk, 0, Kr, Vr, ret, acc, n_rec, 1.1, limit).reshape(n_inst).cpu().numpy()
+    assert kvr.kvr_sketch_device_status(sk) == 0
+    for u in range(n_inst):
+        Ko, Vo, ro, so, to, co, n = orc.swap(Kr_b[u], Vr_b[u], ret_np[u], acc_np[u], s1[u], cells_o[u], n_rec, 1.1, limit,
+                                             seeds, round_rows=rounder)
+        assert n == n_sw[u] == limit
+        assert (ret.reshape(n_inst, -1)[u].cpu().numpy() == ro).all()
+        assert (acc.reshape(n_inst, -1)[u].cpu().numpy() == so).all()
+        assert (ro[:limit] != ret_np[u][:limit]).all()                           # the lowest token indices went
     kvr.kvr_sketch_destroy(sk)
 
 
