@@ -4,52 +4,56 @@
 // row of one head-instance, walks that cell's token list (ascending token index, built once per
 // handle from the hash tables), skips retained tokens by the membership bitmap, and adds
 //     cell.key += K[J],     cell.value += g_i(J) * V[J]
-// in fp32: the even and the odd tokens of the list are summed by different warps, each in ascending
+// in fp32: the tokens of the list are dealt to four half-warps in turn, each summing its own in ascending
 // order (batches of eight rows added plainly, the batch sums accumulated with compensation), and the
-// two sums added at the end.  No atomics: the cells are bit-reproducible.
+// four sums are added in a fixed order at the end.  No atomics: the cells are bit-reproducible.
 #include "kvr_internal.h"
 
 namespace {
 
-constexpr int INS_THREADS = 128;   // warp w: keys (w even) or values (w odd) of every other token of the cell
+constexpr int INS_THREADS = 128;   // warp w: keys (w even) or values (w odd); its two half-warps and the two warps of a kind take every fourth token each
 constexpr int INS_UNROLL = 8;      // rows requested per lane before the first is added
 
 template <typename T>
 __global__ void __launch_bounds__(INS_THREADS)
 insert_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ full_list,
               const int8_t* __restrict__ tok_g, const uint32_t* __restrict__ bitmap_all, int bitmap_words,
-              const uint2* __restrict__ K, const uint2* __restrict__ V, int N, int max_ctx, int b,
+              const uint4* __restrict__ K, const uint4* __restrict__ V, int N, int max_ctx, int b,
               int inst0, int n_tbl, int r, float* __restrict__ cells_all) {
     __shared__ uint32_t s_tok[INS_THREADS];
     __shared__ int s_wcnt[INS_THREADS / 32];
-    __shared__ float4 s_part[2][KVR_D / 4];      // sums of the odd tokens: [keys | values][4 channels]
+    __shared__ float4 s_part[2][KVR_D / 4];      // sums of the tokens 2, 3 (mod 4): [keys | values][4 channels]
 
     const int c = blockIdx.x, i = blockIdx.y, u = blockIdx.z, inst = inst0 + u;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int kv = warp & 1, par = warp >> 1;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, l16 = lane & 15;
+    const int kv = warp & 1, par = (warp >> 1) * 2 + (lane >> 4);             // this half-warp's tokens: par, par + 4, ...
     const uint32_t* bitmap = bitmap_all + (size_t)inst * bitmap_words;
     const int tb = n_tbl > 1 ? inst % n_tbl : 0;              // hash tables of this kv head (seeds per head) or the shared ones
     full_off += (size_t)tb * r * (b + 1);
     const int32_t* list = full_list + ((size_t)tb * r + i) * max_ctx;
     const int8_t* g = tok_g + ((size_t)tb * r + i) * max_ctx;
-    const uint2* src = (kv ? V : K) + (size_t)u * N * (KVR_D / 4) + lane;     // 4 channels (8 bytes) per lane
+    const uint4* src = (kv ? V : K) + (size_t)u * N * (KVR_D / 8) + l16;      // 8 channels (16 bytes) per lane
     const int p0 = full_off[i * (b + 1) + c], p1 = full_off[i * (b + 1) + c + 1];
 
     // Two levels: the rows of one batch (up to INS_UNROLL) are added plainly, in order, and the batch
     // sum goes into a compensated running sum, so the rounding error does not grow with the length
     // of the cell's token list.
-    float s[4] = {0.f, 0.f, 0.f, 0.f}, cc[4] = {0.f, 0.f, 0.f, 0.f}, blk[4] = {0.f, 0.f, 0.f, 0.f};
-    auto add = [&](uint2 x, uint32_t e) {
-        const float2 lo = KvrType<T>::to_f2(x.x), hi = KvrType<T>::to_f2(x.y);
+    float s[8], cc[8], blk[8];
+#pragma unroll
+    for (int d = 0; d < 8; ++d) s[d] = cc[d] = blk[d] = 0.f;
+    auto add = [&](const uint4& x, uint32_t e) {
         const float sg = (kv && (e >> 31)) ? -1.f : 1.f;      // g_i(J) for the values, +1 for the keys
-        blk[0] = fmaf(lo.x, sg, blk[0]);                      // = blk + g v, rounded once
-        blk[1] = fmaf(lo.y, sg, blk[1]);
-        blk[2] = fmaf(hi.x, sg, blk[2]);
-        blk[3] = fmaf(hi.y, sg, blk[3]);
+        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const float2 f = KvrType<T>::to_f2(w[q]);
+            blk[2 * q] = fmaf(f.x, sg, blk[2 * q]);           // = blk + g v, rounded once
+            blk[2 * q + 1] = fmaf(f.y, sg, blk[2 * q + 1]);
+        }
     };
     auto fold = [&]() {
 #pragma unroll
-        for (int d = 0; d < 4; ++d) {
+        for (int d = 0; d < 8; ++d) {
             const float v = blk[d], t = s[d] + v;
             cc[d] += (fabsf(s[d]) >= fabsf(v)) ? (s[d] - t) + v : (v - t) + s[d];
             s[d] = t;
@@ -78,32 +82,43 @@ insert_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ 
         }
         if (keep) s_tok[off + __popc(m & ((1u << lane) - 1u))] = packed;
         __syncthreads();
-        // this warp's tokens of the round: t = par, par + 2, ... (ascending token index)
-        for (int t0 = par; t0 < n; t0 += 2 * INS_UNROLL) {
+        // this half-warp's tokens of the round: t = par, par + 4, ... (ascending token index)
+        for (int t0 = par; t0 < n; t0 += 4 * INS_UNROLL) {
             uint32_t e[INS_UNROLL];
-            uint2 x[INS_UNROLL];
+            uint4 x[INS_UNROLL];
 #pragma unroll
             for (int q = 0; q < INS_UNROLL; ++q) {
-                const int t = t0 + 2 * q;
+                const int t = t0 + 4 * q;
                 e[q] = (t < n) ? s_tok[t] : 0xFFFFFFFFu;
-                if (t < n) x[q] = src[(size_t)(e[q] & 0x7FFFFFFFu) * (KVR_D / 4)];
+                if (t < n) x[q] = src[(size_t)(e[q] & 0x7FFFFFFFu) * (KVR_D / 8)];
             }
-            blk[0] = blk[1] = blk[2] = blk[3] = 0.f;
+#pragma unroll
+            for (int d = 0; d < 8; ++d) blk[d] = 0.f;
 #pragma unroll
             for (int q = 0; q < INS_UNROLL; ++q)
-                if (t0 + 2 * q < n) add(x[q], e[q]);
+                if (t0 + 4 * q < n) add(x[q], e[q]);
             fold();
         }
         __syncthreads();
     }
-    // even tokens + odd tokens, in that order
-    float4 mine = make_float4(s[0] + cc[0], s[1] + cc[1], s[2] + cc[2], s[3] + cc[3]);
-    if (par) s_part[kv][lane] = mine;
+    // (tokens 0 mod 4 + tokens 1 mod 4) + (tokens 2 mod 4 + tokens 3 mod 4), in that order
+    float mine[8];
+#pragma unroll
+    for (int d = 0; d < 8; ++d) {
+        mine[d] = s[d] + cc[d];
+        mine[d] += __shfl_down_sync(0xFFFFFFFFu, mine[d], 16);                  // (meaningful in the lower half-warp)
+    }
+    const bool upper = (warp >> 1) != 0;
+    if (upper && lane < 16) {
+        s_part[kv][2 * l16] = make_float4(mine[0], mine[1], mine[2], mine[3]);
+        s_part[kv][2 * l16 + 1] = make_float4(mine[4], mine[5], mine[6], mine[7]);
+    }
     __syncthreads();
-    if (!par) {
-        const float4 o = s_part[kv][lane];
-        float* cell = cells_all + ((((size_t)inst * 2 + kv) * r + i) * b + c) * KVR_D + 4 * lane;
-        *reinterpret_cast<float4*>(cell) = make_float4(mine.x + o.x, mine.y + o.y, mine.z + o.z, mine.w + o.w);
+    if (!upper && lane < 16) {
+        const float4 o0 = s_part[kv][2 * l16], o1 = s_part[kv][2 * l16 + 1];
+        float* cell = cells_all + ((((size_t)inst * 2 + kv) * r + i) * b + c) * KVR_D + 8 * l16;
+        *reinterpret_cast<float4*>(cell) = make_float4(mine[0] + o0.x, mine[1] + o0.y, mine[2] + o0.z, mine[3] + o0.w);
+        *reinterpret_cast<float4*>(cell + 4) = make_float4(mine[4] + o1.x, mine[5] + o1.y, mine[6] + o1.z, mine[7] + o1.w);
     }
 }
 
@@ -147,12 +162,12 @@ cudaError_t kvr_launch_insert(kvr_sketch* sk, int inst0, int n_inst, int N, cons
     dim3 g(sk->d.b, sk->d.r, n_inst);
     if (sk->d.kv_dtype == KVR_F16)
         insert_kernel<__half><<<g, INS_THREADS, 0, st>>>(sk->full_off, sk->full_list, sk->tok_g, sk->bitmap,
-                                                         sk->bitmap_words, (const uint2*)K, (const uint2*)V,
+                                                         sk->bitmap_words, (const uint4*)K, (const uint4*)V,
                                                          N, sk->d.max_context, sk->d.b, inst0, sk->n_tbl, sk->d.r, sk->cells);
     else
         insert_kernel<__nv_bfloat16><<<g, INS_THREADS, 0, st>>>(sk->full_off, sk->full_list, sk->tok_g, sk->bitmap,
-                                                                sk->bitmap_words, (const uint2*)K,
-                                                                (const uint2*)V, N, sk->d.max_context,
+                                                                sk->bitmap_words, (const uint4*)K,
+                                                                (const uint4*)V, N, sk->d.max_context,
                                                                 sk->d.b, inst0, sk->n_tbl, sk->d.r, sk->cells);
     sk->launches += 1;
     return cudaGetLastError();
