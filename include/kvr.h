@@ -346,12 +346,15 @@ int32_t kvr_last_score_kernel(const kvr_sketch_t* sk);
  * handle so far completed normally; anything else means outputs since then are invalid. */
 kvr_status_t kvr_sketch_device_status(kvr_sketch_t* sk, int32_t* status, void* cuda_stream);
 
-/* Test hook for that give-up path (no counterpart in the paper).  wait_limit_ns replaces the 0.2 s limit
- * (100 us .. 1 s); unannounced_bytes > 0 (a multiple of 16, at most 4096) makes the staged kernel expect
- * that many bytes more on its cells barrier than its copies deliver, so the barrier never completes:
- * every class CTA waits wait_limit_ns, sets bit 0 of the status word and carries on with the cells,
- * which landed long before (the outputs are still right; nothing faults or hangs).  0 bytes and
- * 200 000 000 ns restore normal operation.  Errors: INVALID_ARG. */
+/* Test hook for the give-up paths (no counterpart in the paper).  wait_limit_ns replaces the 0.2 s limit
+ * (100 us .. 1 s); unannounced_bytes > 0 (a multiple of 16, at most 4096) makes a kernel expect that many
+ * bytes more on a staging barrier than its copies deliver, so the barrier never completes:
+ *   - staged decode kernel: every class CTA waits wait_limit_ns on its cells barrier, sets bit 0 of the
+ *     status word and carries on with the cells, which landed long before (the outputs are still right);
+ *   - tcgen05 scoring kernel: the wait for the query tile runs out, the CTA sets bit 1, skips its tiles
+ *     and runs to its end, where it releases its tensor memory (the scores of that compress are void).
+ * Nothing faults or hangs, and no copy is in flight when a CTA exits (the limit cannot be set below the
+ * time a copy takes).  0 bytes and 200 000 000 ns restore normal operation.  Errors: INVALID_ARG. */
 kvr_status_t kvr_sketch_set_wait_test(kvr_sketch_t* sk, int64_t wait_limit_ns, int32_t unannounced_bytes);
 
 /* Algorithm 3 ("insert newly generated token(s) T and compress") as one call.  The caller's exact

@@ -27,7 +27,6 @@ constexpr int TC_TILE_BYTES = 2 * TC_HALF_BYTES;
 constexpr int TC_TMEM_COLS = 256;
 constexpr int TC_DYN_SMEM = (1 + TC_STAGES) * TC_TILE_BYTES + 1024;   // Q + ring + alignment slack
 constexpr unsigned FULL = 0xFFFFFFFFu;
-constexpr unsigned long long TC_WAIT_LIMIT_NS = 200ull * 1000 * 1000;
 
 // barrier indices
 constexpr int B_Q = 0, B_FULL = 1, B_EMPTY = B_FULL + TC_STAGES, B_TFULL = B_EMPTY + TC_STAGES, B_TEMPTY = B_TFULL + 2,
@@ -52,13 +51,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     unsigned long long t0, t;
     asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t0));
     while (!mbar_try_wait(bar, parity)) {
         asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t));
-        if (t - t0 > TC_WAIT_LIMIT_NS) return false;
+        if (t - t0 > limit_ns) return false;
     }
     return true;
 }
@@ -126,7 +125,9 @@ __global__ void __launch_bounds__(TC_THREADS, 2)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, int N, int M,
                 int W, int causal, int chunk, int n_chunks, float scale_log2e,
                 float2* partial /*[u][2 n_chunks][Mpad]: written by pass 1, read by pass 2*/,
-                float* __restrict__ scores_all, int max_ctx, int inst0, int* __restrict__ status) {
+                float* __restrict__ scores_all, int max_ctx, int inst0, int* __restrict__ status,
+                unsigned long long wait_ns /*limit of every mbarrier wait*/,
+                uint32_t tx_extra /*0; a test announces bytes that never arrive, so that the waits run out*/) {
     extern __shared__ unsigned char smem_raw[];
     __shared__ __align__(8) unsigned long long s_bar[B_COUNT];
     __shared__ uint32_t s_tmem;
@@ -170,12 +171,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const uint32_t it0 = (uint32_t)mt * (uint32_t)n_tiles;           // tiles consumed before this m-tile
         if (warp == 0) {
             if (lane == 0 && !gave_up) {
-                mbar_expect_tx(bar(B_Q), TC_TILE_BYTES);
+                mbar_expect_tx(bar(B_Q), TC_TILE_BYTES + tx_extra);
                 tma_load_2d(sQ, &tmQ, 0, u * M + mt * 128, bar(B_Q));
                 tma_load_2d(sQ + TC_HALF_BYTES, &tmQ, 64, u * M + mt * 128, bar(B_Q));
                 for (int i = 0; i < n_tiles; ++i) {
                     const uint32_t it = it0 + i, s = it % TC_STAGES, ph = (it / TC_STAGES) & 1u;
-                    if (!mbar_wait(bar(B_EMPTY + s), ph ^ 1u)) { gave_up = true; break; }
+                    if (!mbar_wait(bar(B_EMPTY + s), ph ^ 1u, wait_ns)) { gave_up = true; break; }
                     mbar_expect_tx(bar(B_FULL + s), TC_TILE_BYTES);
                     const int row = u * N + n_begin + i * TC_NT;
                     tma_load_2d(sK + s * TC_TILE_BYTES, &tmK, 0, row, bar(B_FULL + s));
@@ -184,11 +185,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             }
         } else if (warp == 1) {
             if (lane == 0 && !gave_up) {
-                if (!mbar_wait(bar(B_Q), (uint32_t)mt & 1u)) gave_up = true;
+                if (!mbar_wait(bar(B_Q), (uint32_t)mt & 1u, wait_ns)) gave_up = true;
                 for (int i = 0; i < n_tiles && !gave_up; ++i) {
                     const uint32_t it = it0 + i, s = it % TC_STAGES, ph = (it / TC_STAGES) & 1u;
                     const uint32_t buf = it & 1u, bph = (it >> 1) & 1u;
-                    if (!mbar_wait(bar(B_TEMPTY + buf), bph ^ 1u) || !mbar_wait(bar(B_FULL + s), ph)) { gave_up = true; break; }
+                    if (!mbar_wait(bar(B_TEMPTY + buf), bph ^ 1u, wait_ns) || !mbar_wait(bar(B_FULL + s), ph, wait_ns)) { gave_up = true; break; }
                     tc_fence_after();
 #pragma unroll
                     for (int k = 0; k < 8; ++k) {                       // 8 x 16 channels = the head dimension
@@ -236,7 +237,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 __threadfence_block();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(B_EPI));
-                if (!__all_sync(FULL, mbar_wait(bar(B_EPI), epi_round & 1u))) gave_up = true;
+                if (!__all_sync(FULL, mbar_wait(bar(B_EPI), epi_round & 1u, wait_ns))) gave_up = true;
                 ++epi_round;
                 const float2 a0 = s_stat[0][q * 32 + lane], a1 = s_stat[1][q * 32 + lane];
                 const float mrow = fmaxf(a0.x, a1.x);                    // finite: every row has seen column 0
@@ -247,7 +248,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             }
             for (int i = 0; i < n_tiles && !gave_up; ++i) {
                 const uint32_t it = it0 + i, buf = it & 1u, bph = (it >> 1) & 1u;
-                if (!__all_sync(FULL, mbar_wait(bar(B_TFULL + buf), bph))) { gave_up = true; break; }
+                if (!__all_sync(FULL, mbar_wait(bar(B_TFULL + buf), bph, wait_ns))) { gave_up = true; break; }
                 tc_fence_after();
                 const int n0 = n_begin + i * TC_NT;
                 float vv[2][32];
@@ -301,7 +302,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     __threadfence_block();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar(B_EPI));
-                    if (!__all_sync(FULL, mbar_wait(bar(B_EPI), epi_round & 1u))) { gave_up = true; break; }
+                    if (!__all_sync(FULL, mbar_wait(bar(B_EPI), epi_round & 1u, wait_ns))) { gave_up = true; break; }
                     ++epi_round;
                     const int et = tid - 64;
                     if (et < TC_NT) {
@@ -365,10 +366,10 @@ cudaError_t launch_typed(kvr_sketch* sk, const ScoreShape& s, const CUtensorMap&
     dim3 grid(s.n_chunks, s.n_inst);
     score_tc_kernel<T, 1><<<grid, TC_THREADS, TC_DYN_SMEM, st>>>(tmQ, tmK, s.N, s.M, s.W, s.causal, s.chunk, s.n_chunks, s.scale_log2e,
                                                                  partial, sk->scores, sk->d.max_context,
-                                                                 s.inst0, sk->dev_status);
+                                                                 s.inst0, sk->dev_status, sk->wait_ns, sk->tx_extra);
     score_tc_kernel<T, 2><<<grid, TC_THREADS, TC_DYN_SMEM, st>>>(tmQ, tmK, s.N, s.M, s.W, s.causal, s.chunk, s.n_chunks, s.scale_log2e,
                                                                  partial, sk->scores, sk->d.max_context,
-                                                                 s.inst0, sk->dev_status);
+                                                                 s.inst0, sk->dev_status, sk->wait_ns, sk->tx_extra);
     sk->launches += 2;
     return cudaGetLastError();
 }

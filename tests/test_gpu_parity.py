@@ -10,7 +10,7 @@ import paper_2512_17917_b200 as kvr
 from oracle import kvr_oracle as orc
 from paper_2512_17917_b200 import synth
 
-from kvr_testlib import TOL, dec_to_inst, inst_major, make_case, run_and_check, sampled_instances
+from kvr_testlib import TOL, dec_to_inst, inst_major, make_case, obs_to_inst, run_and_check, sampled_instances
 
 pytestmark = pytest.mark.gpu
 F16, BF16 = torch.float16, torch.bfloat16
@@ -736,6 +736,36 @@ def test_bounded_wait_gives_up_and_reports():
             kvr.kvr_sketch_set_wait_test(sk, 10, 16)                            # a limit that could cut a copy short
         finally:
             kvr.kvr_sketch_destroy(sk)
+
+
+def test_bounded_wait_of_the_scoring_kernel_gives_up_and_reports():
+    """The tcgen05 scoring kernel's waits are bounded too.  With the hook its wait for the query tile
+    runs out: status bit 1, the CTA runs to its end and releases its tensor memory, nothing faults or
+    hangs; with the hook off again the same handle compresses normally and matches the oracle."""
+    seeds = synth.hash_seeds(9200)
+    B, H, Hq, N, W, R, b = 1, 2, 8, 1024, 32, 100, 12
+    K, V, Q, q = make_case(9201, B, H, Hq, N, W, F16, 1)
+    dev = "cuda"
+    sk = kvr.kvr_sketch_create(b=b, batch=B, n_layers=1, n_kv_heads=H, n_q_heads=Hq, max_context=N, kv_dtype=F16,
+                               hash_seeds=seeds)
+    kvr.kvr_sketch_set_score_kernel(sk, kvr.KVR_SCORE_TCGEN05)
+    kvr.kvr_sketch_set_wait_test(sk, 1_000_000, 16)
+    kvr.kvr_compress(sk, 0, K[0].to(dev), V[0].to(dev), Q[0].to(dev), R, 0)
+    assert kvr.kvr_last_score_kernel(sk) == kvr.KVR_SCORE_TCGEN05
+    assert kvr.kvr_sketch_device_status(sk) & 2
+    kvr.kvr_sketch_destroy(sk)
+    # a fresh handle (the status word is sticky), hook set and taken back: normal operation
+    sk = kvr.kvr_sketch_create(b=b, batch=B, n_layers=1, n_kv_heads=H, n_q_heads=Hq, max_context=N, kv_dtype=F16,
+                               hash_seeds=seeds)
+    kvr.kvr_sketch_set_score_kernel(sk, kvr.KVR_SCORE_TCGEN05)
+    kvr.kvr_sketch_set_wait_test(sk, 1_000_000, 16)
+    kvr.kvr_sketch_set_wait_test(sk, 200_000_000, 0)
+    kvr.kvr_compress(sk, 0, K[0].to(dev), V[0].to(dev), Q[0].to(dev), R, 0)
+    assert kvr.kvr_sketch_device_status(sk) == 0
+    got = kvr.kvr_get_scores(sk, 0).reshape(B * H, N).cpu().numpy()
+    want = orc.scores(obs_to_inst(Q[0], H), inst_major(K[0]))
+    kvr.kvr_sketch_destroy(sk)
+    np.testing.assert_allclose(got, want, rtol=2e-4, atol=1e-7)
 
 
 def test_per_layer_budgets_in_one_handle():
