@@ -177,3 +177,89 @@ def run_and_check(K, V, Qobs, q, *, R, n_recent, b, seeds, index_mix=True, layer
     assert np.isfinite(out_g).all() and err <= TOL, err
     kvr.kvr_sketch_destroy(sk)
     return out_g, out_o
+
+
+def run_stream_case(*, which, dtype, one_call, B, H, Hq, N, R, b, n_rec0, r_budget, c_budget, slack, steps, rate, max_swaps,
+                    seed):
+    """A generation loop on the GPU (decode, score accumulation, kvr_append per step) against the oracle's
+    compress_stream, every step and every head-instance.  one_call: the decode call keeps the step's scores
+    (kvr_decode_attention_scored) instead of two accumulate calls after it.  Returns (steps in which the
+    Recent part overflowed, swaps in total)."""
+    G = Hq // H
+    n_inst = B * H
+    seeds = synth.hash_seeds(seed)
+    total = N + sum(steps)
+    K, V, Q, q = make_case(seed + 1, B, H, Hq, total, 8, dtype, 1)
+    dev = "cuda"
+    sk = kvr.kvr_sketch_create(b=b, batch=B, n_layers=1, n_kv_heads=H, n_q_heads=Hq, max_context=total, kv_dtype=dtype,
+                               hash_seeds=seeds)
+    kvr.kvr_sketch_set_decode_kernel(sk, kvr.KVR_DECODE_SPLIT if which == "split" else kvr.KVR_DECODE_STAGED)
+    Kall, Vall = inst_major(K[0]), inst_major(V[0])
+    Kr, Vr, ret = kvr.kvr_compress(sk, 0, K[0, :, :, :N].contiguous().to(dev), V[0, :, :, :N].contiguous().to(dev),
+                                   Q[0].to(dev), R, n_rec0)
+    cmp0 = kvr.kvr_get_assignment(sk, 0)[0].reshape(n_inst, -1).cpu().numpy()
+    s0 = kvr.kvr_get_scores(sk, 0).reshape(n_inst, -1)
+    acc = torch.gather(s0, 1, ret.reshape(n_inst, -1).long()).reshape(B, H, min(R, N)).contiguous()
+    # oracle state per head-instance
+    o_cells = list(orc.insert(Kall[:, :N], Vall[:, :N], cmp0, seeds, b))
+    o_Kr, o_Vr = list(inst_major(Kr).astype(np.float64)), list(inst_major(Vr).astype(np.float64))
+    o_ret = list(ret.reshape(n_inst, -1).cpu().numpy())
+    n_recent, ctx, drops, swaps = n_rec0, N, 0, 0
+    rounder = lambda x: torch.from_numpy(np.asarray(x, np.float64)).to(dtype).double().numpy()
+    ulp = 2.0 ** -11 if dtype == torch.float16 else 2.0 ** -8
+    for it, n_new in enumerate(steps):
+        # ---- decode over the current storage, then the attention mass goes to the scores
+        qd = synth.make_decode_q(seed + 300 + it, B, Hq, 128, dtype, dev)
+        if one_call:
+            out = kvr.kvr_decode_attention_scored(sk, 0, qd, Kr, Vr, ret, acc)
+        else:
+            out = kvr.kvr_decode_attention(sk, 0, qd, Kr, Vr, ret)
+            kvr.kvr_accumulate_scores(sk, 0, qd, Kr, acc)
+            kvr.kvr_accumulate_vague_scores(sk, 0, qd)
+        qo = dec_to_inst(qd, H)
+        want = orc.decode(qo, np.stack(o_Kr), np.stack(o_Vr), np.stack(o_ret), np.stack(o_cells), ctx, seeds)
+        assert np.abs(out.reshape(n_inst, G, 128).cpu().numpy() - want).max() <= TOL
+        tok_g = kvr.kvr_get_scores(sk, 0).reshape(n_inst, -1).cpu().numpy()       # [n_inst, context of the last overflow step]
+        acc_np = acc.reshape(n_inst, -1).cpu().numpy()
+        # ---- Algorithm 3 for the new tokens
+        Kn, Vn = K[0, :, :, ctx:ctx + n_new].contiguous().to(dev), V[0, :, :, ctx:ctx + n_new].contiguous().to(dev)
+        before = n_recent + n_new
+        Kr, Vr, ret, acc, n_recent_g, n_sw = kvr.kvr_append(sk, 0, Kr, Vr, ret, acc, n_recent, Kn, Vn, r_budget, c_budget,
+                                                            slack, rate, max_swaps)
+        assert kvr.kvr_sketch_device_status(sk) == 0
+        n_sw = n_sw.reshape(n_inst).cpu().numpy()
+        ret_g, acc_g = ret.reshape(n_inst, -1).cpu().numpy(), acc.reshape(n_inst, -1).cpu().numpy()
+        cells_g = kvr.kvr_get_cells(sk, 0).reshape(n_inst, 2, 3, b, 128).cpu().numpy().transpose(0, 2, 3, 1, 4)
+        tok_after = kvr.kvr_get_scores(sk, 0).reshape(n_inst, -1).cpu().numpy()
+        for u in range(n_inst):
+            # the oracle steps from its own storage, with the scores the kernels accumulated
+            tok_u = np.concatenate([tok_g[u], np.zeros(ctx + n_new - tok_g.shape[1], np.float32)])   # tokens beyond are rows
+            Ko, Vo, ro, so, rec_o, to, co, n = orc.compress_stream(
+                o_Kr[u], o_Vr[u], o_ret[u], acc_np[u], n_recent, tok_u, o_cells[u], Kall[u, ctx:ctx + n_new],
+                Vall[u, ctx:ctx + n_new], np.arange(ctx, ctx + n_new, dtype=np.int32), r_budget, c_budget, slack, rate,
+                max_swaps, seeds, round_rows=rounder)
+            assert rec_o == n_recent_g and n == n_sw[u]
+            assert (ret_g[u] == ro).all() and (acc_g[u] == so).all()
+            vague = np.setdiff1d(np.arange(ctx + n_new), ro)
+            assert (tok_after[u, vague] == to[vague]).all()
+            # (the tolerance is derived for cells up to about 500 in magnitude and a few updates per cell; a sketch
+            # of a handful of cells sums thousands of tokens per cell, and every swap rounds the cells it touches
+            # to fp32 again, a random walk of half-units in the last place: the bar grows with both)
+            cmax = float(np.abs(co).max())
+            tol = TOL * max(1.0, cmax / 500.0) + np.sqrt(swaps + n + 1.0) * 2.0 ** -22 * cmax
+            err = float(np.abs(cells_g[u] - co).max())
+            assert err <= tol, (err, tol)
+            dk, dv = np.abs(inst_major(Kr)[u] - Ko), np.abs(inst_major(Vr)[u] - Vo)
+            assert (dk <= tol + 2 * ulp * np.abs(Ko)).all() and (dv <= tol + 2 * ulp * np.abs(Vo)).all()
+            # carry the GPU's rows on (a revived row is rounded to the cache type on both sides)
+            o_Kr[u], o_Vr[u], o_ret[u], o_cells[u] = inst_major(Kr)[u].astype(np.float64), inst_major(Vr)[u].astype(np.float64), ro, co
+            swaps += n
+        drops += int(n_recent_g < before)
+        n_recent, ctx = n_recent_g, ctx + n_new
+    # ---- one more decode over the final storage
+    qd = synth.make_decode_q(seed + 999, B, Hq, 128, dtype, dev)
+    out = kvr.kvr_decode_attention(sk, 0, qd, Kr, Vr, ret)
+    want = orc.decode(dec_to_inst(qd, H), np.stack(o_Kr), np.stack(o_Vr), np.stack(o_ret), np.stack(o_cells), ctx, seeds)
+    assert np.abs(out.reshape(n_inst, G, 128).cpu().numpy() - want).max() <= TOL
+    kvr.kvr_sketch_destroy(sk)
+    return drops, swaps

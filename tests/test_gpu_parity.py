@@ -10,7 +10,7 @@ import paper_2512_17917_b200 as kvr
 from oracle import kvr_oracle as orc
 from paper_2512_17917_b200 import synth
 
-from kvr_testlib import TOL, dec_to_inst, inst_major, make_case, obs_to_inst, run_and_check, sampled_instances
+from kvr_testlib import TOL, dec_to_inst, inst_major, make_case, obs_to_inst, run_and_check, run_stream_case, sampled_instances
 
 pytestmark = pytest.mark.gpu
 F16, BF16 = torch.float16, torch.bfloat16
@@ -448,86 +448,19 @@ def test_swap_loop_with_equal_candidate_scores():
     kvr.kvr_sketch_destroy(sk)
 
 
-@pytest.mark.parametrize("which,dtype", [("staged", F16), ("split", BF16)])
-def test_append_runs_algorithm_3_over_several_slack_periods(which, dtype):
+@pytest.mark.parametrize("which,dtype,one_call", [("staged", F16, False), ("split", BF16, False), ("staged", BF16, True),
+                                                  ("split", F16, True)])
+def test_append_runs_algorithm_3_over_several_slack_periods(which, dtype, one_call):
     """kvr_append against the oracle's compress_stream: a generation loop of decode, score
-    accumulation (stored rows and vague tokens) and one kvr_append per step, through more than three
-    Slack periods.  Which rows stay and which tokens are swapped are integer decisions taken in fp32
-    from the scores the kernels accumulated, so row indices, row scores and per-token scores are
-    compared exactly; cells and rows within the tolerance; the decode of every step is compared with
-    the oracle on the storage of that step."""
-    B, H, Hq, N, R, b, n_rec0 = 1, 2, 8, 1000, 120, 30, 10
-    G = Hq // H
-    r_budget, c_budget, slack = 10, 110, 6
-    n_inst = B * H
-    seeds = synth.hash_seeds(4711)
-    steps = [3, 1, 2, 4, 1, 3, 2, 2, 4, 1, 3, 2]
-    total = N + sum(steps)
-    K, V, Q, q = make_case(4712, B, H, Hq, total, 8, dtype, 1)
-    dev = "cuda"
-    sk = kvr.kvr_sketch_create(b=b, batch=B, n_layers=1, n_kv_heads=H, n_q_heads=Hq, max_context=total, kv_dtype=dtype,
-                               hash_seeds=seeds)
-    kvr.kvr_sketch_set_decode_kernel(sk, kvr.KVR_DECODE_SPLIT if which == "split" else kvr.KVR_DECODE_STAGED)
-    Kall, Vall = inst_major(K[0]), inst_major(V[0])
-    Kr, Vr, ret = kvr.kvr_compress(sk, 0, K[0, :, :, :N].contiguous().to(dev), V[0, :, :, :N].contiguous().to(dev),
-                                   Q[0].to(dev), R, n_rec0)
-    cmp0 = kvr.kvr_get_assignment(sk, 0)[0].reshape(n_inst, -1).cpu().numpy()
-    s0 = kvr.kvr_get_scores(sk, 0).reshape(n_inst, -1)
-    acc = torch.gather(s0, 1, ret.reshape(n_inst, -1).long()).reshape(B, H, R).contiguous()
-    # oracle state per head-instance
-    o_cells = list(orc.insert(Kall[:, :N], Vall[:, :N], cmp0, seeds, b))
-    o_Kr, o_Vr = list(inst_major(Kr).astype(np.float64)), list(inst_major(Vr).astype(np.float64))
-    o_ret = list(ret.reshape(n_inst, -1).cpu().numpy())
-    n_recent, ctx, drops, swaps = n_rec0, N, 0, 0
-    rounder = lambda x: torch.from_numpy(np.asarray(x, np.float64)).to(dtype).double().numpy()
-    ulp = 2.0 ** -11 if dtype == F16 else 2.0 ** -8
-    for it, n_new in enumerate(steps):
-        # ---- decode over the current storage, then the attention mass goes to the scores
-        qd = synth.make_decode_q(5000 + it, B, Hq, 128, dtype, dev)
-        out = kvr.kvr_decode_attention(sk, 0, qd, Kr, Vr, ret)
-        kvr.kvr_accumulate_scores(sk, 0, qd, Kr, acc)
-        kvr.kvr_accumulate_vague_scores(sk, 0, qd)
-        qo = dec_to_inst(qd, H)
-        want = orc.decode(qo, np.stack(o_Kr), np.stack(o_Vr), np.stack(o_ret), np.stack(o_cells), ctx, seeds)
-        assert np.abs(out.reshape(n_inst, G, 128).cpu().numpy() - want).max() <= TOL
-        tok_g = kvr.kvr_get_scores(sk, 0).reshape(n_inst, -1).cpu().numpy()       # [n_inst, context of the last overflow step]
-        acc_np = acc.reshape(n_inst, -1).cpu().numpy()
-        # ---- Algorithm 3 for the new tokens
-        Kn, Vn = K[0, :, :, ctx:ctx + n_new].contiguous().to(dev), V[0, :, :, ctx:ctx + n_new].contiguous().to(dev)
-        before = n_recent + n_new
-        Kr, Vr, ret, acc, n_recent_g, n_sw = kvr.kvr_append(sk, 0, Kr, Vr, ret, acc, n_recent, Kn, Vn, r_budget, c_budget,
-                                                            slack, 1.1, 20)
-        assert kvr.kvr_sketch_device_status(sk) == 0
-        n_sw = n_sw.reshape(n_inst).cpu().numpy()
-        ret_g, acc_g = ret.reshape(n_inst, -1).cpu().numpy(), acc.reshape(n_inst, -1).cpu().numpy()
-        cells_g = kvr.kvr_get_cells(sk, 0).reshape(n_inst, 2, 3, b, 128).cpu().numpy().transpose(0, 2, 3, 1, 4)
-        tok_after = kvr.kvr_get_scores(sk, 0).reshape(n_inst, -1).cpu().numpy()
-        for u in range(n_inst):
-            # the oracle steps from its own storage, with the scores the kernels accumulated
-            tok_u = np.concatenate([tok_g[u], np.zeros(ctx + n_new - tok_g.shape[1], np.float32)])   # tokens beyond are rows
-            Ko, Vo, ro, so, rec_o, to, co, n = orc.compress_stream(
-                o_Kr[u], o_Vr[u], o_ret[u], acc_np[u], n_recent, tok_u, o_cells[u], Kall[u, ctx:ctx + n_new],
-                Vall[u, ctx:ctx + n_new], np.arange(ctx, ctx + n_new, dtype=np.int32), r_budget, c_budget, slack, 1.1, 20,
-                seeds, round_rows=rounder)
-            assert rec_o == n_recent_g and n == n_sw[u]
-            assert (ret_g[u] == ro).all() and (acc_g[u] == so).all()
-            vague = np.setdiff1d(np.arange(ctx + n_new), ro)
-            assert (tok_after[u, vague] == to[vague]).all()
-            assert np.abs(cells_g[u] - co).max() <= TOL
-            dk, dv = np.abs(inst_major(Kr)[u] - Ko), np.abs(inst_major(Vr)[u] - Vo)
-            assert (dk <= TOL + 2 * ulp * np.abs(Ko)).all() and (dv <= TOL + 2 * ulp * np.abs(Vo)).all()
-            # carry the GPU's rows on (a revived row is rounded to the cache type on both sides)
-            o_Kr[u], o_Vr[u], o_ret[u], o_cells[u] = inst_major(Kr)[u].astype(np.float64), inst_major(Vr)[u].astype(np.float64), ro, co
-            swaps += n
-        drops += int(n_recent_g < before)
-        n_recent, ctx = n_recent_g, ctx + n_new
+    accumulation (stored rows and vague tokens; as three calls, or kept by the decode call itself) and
+    one kvr_append per step, through more than three Slack periods.  Which rows stay and which tokens
+    are swapped are integer decisions taken in fp32 from the scores the kernels accumulated, so row
+    indices, row scores and per-token scores are compared exactly; cells and rows within the tolerance;
+    the decode of every step is compared with the oracle on the storage of that step."""
+    drops, swaps = run_stream_case(which=which, dtype=dtype, one_call=one_call, B=1, H=2, Hq=8, N=1000, R=120, b=30, n_rec0=10,
+                                   r_budget=10, c_budget=110, slack=6, steps=[3, 1, 2, 4, 1, 3, 2, 2, 4, 1, 3, 2], rate=1.1,
+                                   max_swaps=20, seed=4711)
     assert drops >= 3 and swaps > 0
-    # ---- one more decode over the final storage
-    qd = synth.make_decode_q(5999, B, Hq, 128, dtype, dev)
-    out = kvr.kvr_decode_attention(sk, 0, qd, Kr, Vr, ret)
-    want = orc.decode(dec_to_inst(qd, H), np.stack(o_Kr), np.stack(o_Vr), np.stack(o_ret), np.stack(o_cells), ctx, seeds)
-    assert np.abs(out.reshape(n_inst, G, 128).cpu().numpy() - want).max() <= TOL
-    kvr.kvr_sketch_destroy(sk)
 
 
 @pytest.mark.parametrize("Qn,dtype,causal,b,N0,R", [
@@ -766,6 +699,57 @@ def test_bounded_wait_of_the_scoring_kernel_gives_up_and_reports():
     want = orc.scores(obs_to_inst(Q[0], H), inst_major(K[0]))
     kvr.kvr_sketch_destroy(sk)
     np.testing.assert_allclose(got, want, rtol=2e-4, atol=1e-7)
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_valid_shapes(seed):
+    """Shapes, budgets, widths, types, kernels and options drawn at random (seeded) from everything the
+    library accepts, each through every stage against the oracle: the cases nobody thought of."""
+    rng = np.random.default_rng(1000 + seed)
+    L, B = int(rng.choice([1, 1, 2])), int(rng.choice([1, 1, 2, 3]))
+    H, G = int(rng.choice([1, 2, 3, 4, 8])), int(rng.choice([1, 2, 4, 4, 8]))
+    N = int(rng.integers(*[(1, 40), (40, 700), (700, 4000), (4000, 9000)][int(rng.choice([0, 1, 1, 2, 2, 2, 3]))]))
+    W = int(rng.choice([1, 3, 8, 32, 40]))
+    R = [0, N, N + 5, int(rng.integers(0, N + 1)), int(rng.integers(0, N + 1)), int(rng.integers(0, N + 1))][int(rng.integers(0, 6))]
+    Rr = min(R, N)
+    n_recent = int(rng.integers(0, Rr + 1)) if rng.integers(0, 2) else min(Rr, int(rng.integers(0, 17)))
+    b = int(rng.choice([1, 2, 7, 16, 64, 137, 273, 300])) if rng.integers(0, 2) else int(rng.integers(1, 301))
+    dtype = F16 if rng.integers(0, 2) else BF16
+    r = int(rng.choice([3, 3, 3, 3, 1, 5]))
+    dk = int(rng.choice([kvr.KVR_DECODE_AUTO, kvr.KVR_DECODE_AUTO, kvr.KVR_DECODE_SPLIT, kvr.KVR_DECODE_STAGED]))
+    if (r != 3 or G > 4 or R >= N) and dk == kvr.KVR_DECODE_STAGED:
+        dk = kvr.KVR_DECODE_AUTO                                 # (the staged kernel does not serve these: the call would use the other)
+    sck = int(rng.choice([kvr.KVR_SCORE_AUTO, kvr.KVR_SCORE_AUTO, kvr.KVR_SCORE_MMA_SYNC]))
+    causal = bool(rng.integers(0, 4) == 0) and W <= N
+    combine = "mean" if (rng.integers(0, 5) == 0 and r == 3) else "median"
+    mix = bool(rng.integers(0, 6) != 0)
+    K, V, Q, q = make_case(3000 + seed, B, H, H * G, N, W, dtype, L)
+    seeds = synth.hash_seeds(77 + seed, r) if mix else synth.injective_seeds(r)
+    run_and_check(K, V, Q, q, R=R, n_recent=n_recent, b=b, seeds=seeds, index_mix=mix,
+                  layer_mode="all" if rng.integers(0, 2) else "per_layer", decode_kernel=dk, score_kernel=sck,
+                  obs_causal=causal, combine=combine)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_generation_loops(seed):
+    """The same for the streaming side: random storage sizes, Slack, ReplaceRate (below one too), swap
+    limits and step sizes, as three calls or with the decode call that keeps the scores.  (Sketches of
+    at least 8 cells per row: a swap deletes a queried vector, which carries the rounding error of the
+    cells it was read from, from all three of them, so dozens of swaps on the same two or three cells
+    double a last-place difference between fp32 and fp64 cells again and again.  That is the
+    conditioning of the method on such a sketch, in any precision, not something a tolerance describes.)"""
+    rng = np.random.default_rng(2000 + seed)
+    H, G, B = int(rng.choice([1, 2, 3])), int(rng.choice([1, 2, 4, 8])), int(rng.choice([1, 2]))
+    N = int(rng.integers(60, 2500))
+    r_budget = int(rng.integers(1, 40))
+    R = min(N, r_budget + int(rng.integers(1, max(2, N // 3))))
+    n_rec0 = min(r_budget, R - 1)
+    run_stream_case(which="split" if G == 8 or rng.integers(0, 3) == 0 else "staged", dtype=F16 if rng.integers(0, 2) else BF16,
+                    one_call=bool(rng.integers(0, 2)), B=B, H=H, Hq=H * G, N=N, R=R, b=int(rng.integers(8, 120)), n_rec0=n_rec0,
+                    r_budget=r_budget, c_budget=R - n_rec0, slack=int(rng.integers(0, 9)),
+                    steps=[int(x) for x in rng.integers(1, 6, size=int(rng.integers(3, 10)))],
+                    rate=float(rng.choice([1.1, 1.0, 1.5, 0.9])), max_swaps=int(rng.choice([0, 1, 5, 20, 300, 600])),
+                    seed=9000 + 7 * seed)
 
 
 def test_per_layer_budgets_in_one_handle():
