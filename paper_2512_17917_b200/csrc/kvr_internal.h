@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
 #include <vector>
 
 #include "kvr.h"
@@ -228,6 +229,14 @@ template <> struct KvrType<__nv_bfloat16> {
     static __device__ __forceinline__ __nv_bfloat16 from_float(float x) { return __float2bfloat16_rn(x); }
 };
 
+// Programmatic dependent launch inside one call (the kernels of a compress follow one another on one
+// stream): a kernel lets its successor be scheduled as soon as every CTA has started (or exited), so the
+// successor's CTAs take over the SMs as they become free and run whatever does not depend on the
+// predecessor; before the first access that does, they wait for the predecessor to be complete and
+// its writes to be visible.  Both instructions do nothing in a launch without the attribute.
+__device__ __forceinline__ void kvr_pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
+__device__ __forceinline__ void kvr_pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+
 // element-wise middle of three
 __device__ __forceinline__ float kvr_med3(float x, float y, float z) {
     return fmaxf(fminf(x, y), fminf(fmaxf(x, y), z));
@@ -235,5 +244,23 @@ __device__ __forceinline__ float kvr_med3(float x, float y, float z) {
 // what Algorithm 2 makes of a token's three collected numbers: their middle (the paper), or their mean
 __device__ __forceinline__ float kvr_comb3(float x, float y, float z, int mean) {
     return mean ? (x + y + z) * (1.0f / 3.0f) : kvr_med3(x, y, z);
+}
+// Launch `kern` on `st`; dependent = true: as a programmatic dependent of the kernel launched before it
+// on that stream (see kvr_pdl_trigger / kvr_pdl_wait: the kernel must wait before it touches anything
+// its predecessor writes).
+template <typename... KArgs, typename... Args>
+inline cudaError_t kvr_launch_after(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                    bool dependent, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
 }
 #endif

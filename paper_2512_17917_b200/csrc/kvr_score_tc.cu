@@ -136,6 +136,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int u = blockIdx.y, ck = blockIdx.x;
+    kvr_pdl_trigger();         // the next kernel of the compress may take over SMs as they become free
     const int m_tiles = (M + 127) / 128, Mpad = m_tiles * 128;
     const int n_begin = ck * chunk, n_end = min(n_begin + chunk, N);
     const int n_tiles = (n_end - n_begin + TC_NT - 1) / TC_NT;
@@ -215,6 +216,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 // pair each, 16 loads in flight, then exchange through shared memory; both add the two
                 // halves in the same order, so they hold identical statistics.  (Every CTA of the
                 // head-instance repeats this while its first key tiles are on their way.)
+                // (pass 2 is launched as a programmatic dependent of pass 1: its loads and its first tiles
+                // run beside pass 1's last CTAs; what pass 1 wrote is needed from here on)
+                kvr_pdl_wait();
                 const float2* pp = partial + (size_t)u * 2 * n_chunks * Mpad + row;
                 const int n_parts = 2 * n_chunks;
                 float mx = -INFINITY, l = 0.f;
@@ -367,11 +371,13 @@ cudaError_t launch_typed(kvr_sketch* sk, const ScoreShape& s, const CUtensorMap&
     score_tc_kernel<T, 1><<<grid, TC_THREADS, TC_DYN_SMEM, st>>>(tmQ, tmK, s.N, s.M, s.W, s.causal, s.chunk, s.n_chunks, s.scale_log2e,
                                                                  partial, sk->scores, sk->d.max_context,
                                                                  s.inst0, sk->dev_status, sk->wait_ns, sk->tx_extra);
-    score_tc_kernel<T, 2><<<grid, TC_THREADS, TC_DYN_SMEM, st>>>(tmQ, tmK, s.N, s.M, s.W, s.causal, s.chunk, s.n_chunks, s.scale_log2e,
-                                                                 partial, sk->scores, sk->d.max_context,
-                                                                 s.inst0, sk->dev_status, sk->wait_ns, sk->tx_extra);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    e = kvr_launch_after(score_tc_kernel<T, 2>, grid, dim3(TC_THREADS), TC_DYN_SMEM, st, true, tmQ, tmK, s.N, s.M, s.W, s.causal,
+                         s.chunk, s.n_chunks, s.scale_log2e, partial, sk->scores, sk->d.max_context, s.inst0, sk->dev_status,
+                         sk->wait_ns, sk->tx_extra);
     sk->launches += 2;
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace

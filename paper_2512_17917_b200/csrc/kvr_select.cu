@@ -54,6 +54,8 @@ select_kernel(const float* __restrict__ scores_all, int max_ctx, int inst0, int 
     uint32_t* bitmap = bitmap_all + (size_t)inst * bitmap_words;
     int32_t* ret = ret_out ? ret_out + (size_t)u * R : nullptr;
 
+    kvr_pdl_trigger();
+    kvr_pdl_wait();                      // (as a dependent of the scoring kernel: its scores are complete from here on)
     const int n_cand = N - n_recent;
     const int k = R - n_recent;          // candidates to keep, 0 <= k <= n_cand
     const int rows_cta = ((N + 31) / 32 + SEL_CL - 1) / SEL_CL;
@@ -203,6 +205,8 @@ __global__ void gather_kernel(const uint4* __restrict__ K, const uint4* __restri
     const int u = blockIdx.y;
     const int row = blockIdx.x * (blockDim.x >> 4) + (threadIdx.x >> 4);
     const int c = threadIdx.x & 15;
+    kvr_pdl_trigger();
+    kvr_pdl_wait();                      // (as a dependent of the selection: the index list is complete from here on)
     if (row >= R) return;
     const int J = ret_idx[(size_t)u * R + row];
     const size_t src = ((size_t)u * N + J) * 16 + c, dst = ((size_t)u * R + row) * 16 + c;
@@ -214,10 +218,12 @@ __global__ void gather_kernel(const uint4* __restrict__ K, const uint4* __restri
 
 cudaError_t kvr_launch_select(kvr_sketch* sk, int inst0, int n_inst, int N, int R, int n_recent,
                               int32_t* ret_idx, cudaStream_t st) {
-    select_kernel<<<dim3(SEL_CL, n_inst), SEL_THREADS, 0, st>>>(sk->scores, sk->d.max_context, inst0, N, R, n_recent,
-                                                  ret_idx, sk->cmp_idx, sk->bitmap, sk->bitmap_words);
+    // (follows the scoring kernels of the same compress on `st`)
+    const cudaError_t e = kvr_launch_after(select_kernel, dim3(SEL_CL, n_inst), dim3(SEL_THREADS), 0, st, true, (const float*)sk->scores,
+                                           sk->d.max_context, inst0, N, R, n_recent, ret_idx, sk->cmp_idx, sk->bitmap,
+                                           sk->bitmap_words);
     sk->launches += 1;
-    return cudaGetLastError();
+    return e;
 }
 
 // The same selection on caller-provided scores of `n` stored rows (stride n): positions kept
@@ -233,7 +239,8 @@ cudaError_t kvr_launch_gather(kvr_sketch* sk, int n_inst, int N, int R, const vo
                               const int32_t* ret_idx, void* Kr, void* Vr, cudaStream_t st) {
     if (R <= 0) return cudaSuccess;
     dim3 g((R + 15) / 16, n_inst);
-    gather_kernel<<<g, 256, 0, st>>>((const uint4*)K, (const uint4*)V, ret_idx, N, R, (uint4*)Kr, (uint4*)Vr);
+    const cudaError_t e = kvr_launch_after(gather_kernel, g, dim3(256), 0, st, true, (const uint4*)K, (const uint4*)V, ret_idx, N, R,
+                                           (uint4*)Kr, (uint4*)Vr);
     sk->launches += 1;
-    return cudaGetLastError();
+    return e;
 }

@@ -34,6 +34,8 @@ insert_kernel(const int32_t* __restrict__ full_off, const int32_t* __restrict__ 
     const int8_t* g = tok_g + ((size_t)tb * r + i) * max_ctx;
     const uint4* src = (kv ? V : K) + (size_t)u * N * (KVR_D / 8) + l16;      // 8 channels (16 bytes) per lane
     const int p0 = full_off[i * (b + 1) + c], p1 = full_off[i * (b + 1) + c + 1];
+    kvr_pdl_trigger();
+    kvr_pdl_wait();            // (as a dependent of the kernel before it: the membership bitmap is complete from here on)
 
     // Two levels: the rows of one batch (up to INS_UNROLL) are added plainly, in order, and the batch
     // sum goes into a compensated running sum, so the rounding error does not grow with the length
@@ -160,17 +162,18 @@ __global__ void reconstruct_kernel(const float* __restrict__ cells_all, const in
 cudaError_t kvr_launch_insert(kvr_sketch* sk, int inst0, int n_inst, int N, const void* K, const void* V,
                               cudaStream_t st) {
     dim3 g(sk->d.b, sk->d.r, n_inst);
+    // (follows the copy of the retained rows, or the selection, of the same compress on `st`)
+    cudaError_t e;
     if (sk->d.kv_dtype == KVR_F16)
-        insert_kernel<__half><<<g, INS_THREADS, 0, st>>>(sk->full_off, sk->full_list, sk->tok_g, sk->bitmap,
-                                                         sk->bitmap_words, (const uint4*)K, (const uint4*)V,
-                                                         N, sk->d.max_context, sk->d.b, inst0, sk->n_tbl, sk->d.r, sk->cells);
+        e = kvr_launch_after(insert_kernel<__half>, g, dim3(INS_THREADS), 0, st, true, (const int32_t*)sk->full_off,
+                             (const int32_t*)sk->full_list, (const int8_t*)sk->tok_g, (const uint32_t*)sk->bitmap, sk->bitmap_words,
+                             (const uint4*)K, (const uint4*)V, N, sk->d.max_context, sk->d.b, inst0, sk->n_tbl, sk->d.r, sk->cells);
     else
-        insert_kernel<__nv_bfloat16><<<g, INS_THREADS, 0, st>>>(sk->full_off, sk->full_list, sk->tok_g, sk->bitmap,
-                                                                sk->bitmap_words, (const uint4*)K,
-                                                                (const uint4*)V, N, sk->d.max_context,
-                                                                sk->d.b, inst0, sk->n_tbl, sk->d.r, sk->cells);
+        e = kvr_launch_after(insert_kernel<__nv_bfloat16>, g, dim3(INS_THREADS), 0, st, true, (const int32_t*)sk->full_off,
+                             (const int32_t*)sk->full_list, (const int8_t*)sk->tok_g, (const uint32_t*)sk->bitmap, sk->bitmap_words,
+                             (const uint4*)K, (const uint4*)V, N, sk->d.max_context, sk->d.b, inst0, sk->n_tbl, sk->d.r, sk->cells);
     sk->launches += 1;
-    return cudaGetLastError();
+    return e;
 }
 
 cudaError_t kvr_launch_reconstruct(const kvr_sketch* sk, int inst0, int n_inst, int a, float* Kt, float* Vt,
