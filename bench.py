@@ -599,6 +599,8 @@ def main():
                          "(an option of the library; shows the launch time without the min/max arithmetic)")
     ap.add_argument("--decode-kernel", default="auto", choices=["auto", "split", "staged"],
                     help="force one of the two decode kernels (default: the library chooses)")
+    ap.add_argument("--structured", action="store_true",
+                    help="inputs with four sink tokens per head (peaked scores) instead of plain Gaussian keys")
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu dram bytes per decode launch to report in roofline.traffic (from profiles/)")
     args = ap.parse_args()
@@ -626,6 +628,8 @@ def main():
         w = dataclasses.replace(w, n_layers=args.layers or w.n_layers, decode_steps=args.decode_steps or w.decode_steps,
                                 name=f"{w.name}[layers={args.layers or w.n_layers},decode_steps={args.decode_steps or w.decode_steps}]")
 
+    if args.structured:
+        w = dataclasses.replace(w, structured=True, name=f"{w.name}[sink tokens]")
     if args.preset == "paper":
         ratio = args.budget_ratio or w.budget_ratio
         if args.impl == "reference":

@@ -9,6 +9,8 @@ are datasets this repository does not contain; the Mathematical Analysis section
 i.i.d. normal Q, K, V "with the exception of a few outliers"):
   * K, V ~ N(0, 1) i.i.d.; per (layer, kv head) four distinct key channels are scaled by 8.
   * observation queries and decode queries ~ N(0, 1).
+  * optional structured variant: four sink tokens per (batch, kv head) that every observation query
+    scores far above the rest (plant_sinks), for peaked score distributions.
   * everything is drawn in fp32 by a seeded torch generator on the requested device and rounded
     once to fp16 / bf16; the same bytes go to both sides of a parity test.
   * hash seeds A, A' in [1, p), C, C' in [0, p), p = 2^31 - 1, from numpy's default_rng.
@@ -42,6 +44,7 @@ class Workload:
     n_recent: int = 0         # rows of the budget that are the newest tokens (Recent part)
     budget_rows: int = -1     # explicit exact rows / sketch width (a storage-split preset); -1: from the ratios
     b_cells: int = -1
+    structured: bool = False  # sink tokens planted (plant_sinks)
 
     @property
     def budget(self) -> int:
@@ -135,11 +138,28 @@ def make_decode_q(seed: int, batch: int, n_q_heads: int, D: int, dtype: torch.dt
                        dtype=torch.float32).to(dtype)
 
 
+def plant_sinks(K: torch.Tensor, Qobs: torch.Tensor, n_sink: int = 4, scale: float = 64.0) -> torch.Tensor:
+    """The structured variant of the recipe: attention in real models is peaked (a few "sink" tokens
+    take most of the mass), which i.i.d. Gaussian keys never are.  The keys of the first `n_sink`
+    tokens of every (batch, kv head) become `scale` x the mean of that head's observation-query rows,
+    so every observation query scores them far above the rest (with the defaults the four of them
+    take a quarter to a half of a query's softmax over thousands of tokens).
+    K [batch, H, N, D], Qobs [batch, Hq, W, D]; returns K (changed in place)."""
+    B, H, N, D = K.shape
+    Hq, W = Qobs.shape[1], Qobs.shape[2]
+    mean = Qobs.float().reshape(B, H, (Hq // H) * W, D).mean(dim=2)           # [B, H, D]
+    n = min(n_sink, N)
+    K[:, :, :n, :] = (scale * mean).to(K.dtype)[:, :, None, :]
+    return K
+
+
 def layer_inputs(w: Workload, layer: int, device="cpu"):
     """K, V, Qobs of one layer of a workload (seed = workload seed + 101 x layer)."""
     s = w.seed + 101 * layer
     K, V = make_kv(s, w.batch, w.n_kv_heads, w.context, w.head_dim, w.torch_dtype, device)
     Q = make_queries(s + 1, w.batch, w.n_q_heads, w.obs_window, w.head_dim, w.torch_dtype, device)
+    if w.structured:
+        plant_sinks(K, Q)
     return K, V, Q
 
 

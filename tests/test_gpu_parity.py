@@ -701,6 +701,27 @@ def test_bounded_wait_of_the_scoring_kernel_gives_up_and_reports():
     np.testing.assert_allclose(got, want, rtol=2e-4, atol=1e-7)
 
 
+@pytest.mark.parametrize("dtype,score_kernel", [(F16, kvr.KVR_SCORE_TCGEN05), (BF16, kvr.KVR_SCORE_MMA_SYNC)])
+def test_peaked_scores_with_sink_tokens(dtype, score_kernel):
+    """The structured inputs: four sink tokens per head take a large part of every observation query's softmax
+    (a quarter to a half of it on 4 of 3000 tokens), and decode
+    queries that look at them too.  Every stage against the oracle; the sinks must be retained."""
+    L, B, H, Hq, N, W = 1, 2, 2, 8, 3000, 32
+    K, V, Q, q = make_case(6100, B, H, Hq, N, W, dtype, L)
+    for layer in range(L):
+        synth.plant_sinks(K[layer], Q[layer])
+    mean = Q[0].float().reshape(B, H, (Hq // H) * W, 128).mean(dim=2)                      # decode queries lean the same way
+    q = (q.float() + 3.0 * mean.repeat_interleave(Hq // H, dim=1)[None]).to(dtype)
+    out_g, out_o = run_and_check(K, V, Q, q, R=300, n_recent=16, b=20, seeds=synth.hash_seeds(6101), score_kernel=score_kernel)
+    sk = kvr.kvr_sketch_create(b=20, batch=B, n_layers=1, n_kv_heads=H, n_q_heads=Hq, max_context=N, kv_dtype=dtype,
+                               hash_seeds=synth.hash_seeds(6101))
+    _, _, ret = kvr.kvr_compress(sk, 0, K[0].cuda(), V[0].cuda(), Q[0].cuda(), 300, 16)
+    s = kvr.kvr_get_scores(sk, 0).reshape(B * H, N)
+    assert (ret.reshape(B * H, -1)[:, :4].cpu() == torch.arange(4)).all()                    # the sinks are kept
+    assert (s[:, :4].sum(dim=1) > 0.2 * s.sum(dim=1)).all()                                  # and hold a large part of the mass (4 of 3000 tokens)
+    kvr.kvr_sketch_destroy(sk)
+
+
 @pytest.mark.parametrize("seed", range(16))
 def test_random_valid_shapes(seed):
     """Shapes, budgets, widths, types, kernels and options drawn at random (seeded) from everything the
