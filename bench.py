@@ -430,6 +430,15 @@ def run_stream(args, w):
 
 
 # ------------------------------------------------------------------- several queries per head
+def mq_launches(rows: int) -> int:
+    """Launches of one multi-query call: 64, 32 or 16 query rows per launch, as many as are left."""
+    n = 0
+    while rows > 0:
+        rows -= 64 if rows > 32 else 32 if rows > 16 else 16
+        n += 1
+    return n
+
+
 def run_mq(args, w):
     """--queries Qn: decode attention for Qn queries per head per call (kvr_decode_attention_mq) over the
     compressed cache of the workload, one call per layer, all layers and decode steps replayed from a
@@ -498,7 +507,7 @@ def run_mq(args, w):
            "dtype": "f32 accumulate, f16 hi+lo operands", "data": "synthetic",
            "config": dict(config_of(w), queries_per_head=Qn, decode_steps_per_step=S, launch="per_layer_cuda_graph"),
            "decode_kernel": "decode_mq_kernel", "layer_call_us": round(call_us, 2),
-           "launches_per_layer_call": (Hq // H * Qn + 15) // 16,
+           "launches_per_layer_call": mq_launches(Hq // H * Qn),
            "roofline": {"kernel": "decode_mq_kernel", "bound": "hbm", "achieved": round(bytes_call / (call_us * 1e-6) / 1e9, 1),
                         "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                         "frac": round(bytes_call / (call_us * 1e-6) / 1e9 / peak, 4), "bytes_per_launch": bytes_call,

@@ -2,7 +2,10 @@
 // Algorithm 4 (Revive) fused with p = Softmax(q K^T / sqrt(d_k)), out = p V of the Calculation Phase,
 // where the cost of Algorithm 2's reconstruction is shared by all queries.
 //
-// Up to 16 query rows (query heads of one kv head x queries) are served per launch.  As in the staged
+// Up to 64 query rows (query heads of one kv head x queries) are served per launch, 16 per warp: the
+// warps of a CTA form teams of MT = 1, 2 or 4 that share one tile of reconstructed tokens (each
+// warp reconstructs its part of the tile, then runs the contractions for its own 16 rows), so a
+// token is reconstructed once for all rows of the launch.  As in the staged
 // single-query kernel, a CTA serves (a slice of) one class of compressed tokens with the class's
 // row-1 and row-2 cells staged in shared memory, and a group of 16 lanes reconstructs one token at a
 // time (8 channels per lane, the row-0 cell of the current run in registers).  What differs is what
@@ -151,13 +154,23 @@ __device__ __forceinline__ uint32_t to_h2(uint32_t u) {
     }
 }
 
-template <typename T>
+template <typename T, int MT>
 __global__ void __launch_bounds__(MQ_THREADS, 1)
 decode_mq_kernel(const MqParams p) {
+    constexpr int TPH = 4;                              // tokens a group of 16 lanes reconstructs per tile
+    constexpr int TT = MQ_TILE * MT;                    // tokens of a team's tile: every warp fills 8 slots of it
+    constexpr uint32_t TEAM_TILE_BYTES = (uint32_t)MT * MQ_TILE_BYTES;
+    constexpr int NTEAMS = MQ_WARPS / MT, ROWS_L = MQ_ROWS * MT;
     extern __shared__ __align__(16) unsigned char smem[];
     const MqLayout L = mq_layout(p.n1, p.lcap);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, gw = lane >> 4, lg = lane & 15;
     const int grp = warp * 2 + gw;
+    const int team = warp / MT, wt = warp % MT, hw = wt * 2 + gw;      // team, warp in team (= its 16 rows), group in team
+    const int rowbase = p.row0 + wt * MQ_ROWS;
+    auto team_sync = [&]() {
+        if constexpr (MT == 1) __syncwarp();
+        else asm volatile("bar.sync %0, %1;\n" ::"r"(1 + team), "r"(32 * MT) : "memory");
+    };
     const int fg = lane >> 2, ft = lane & 3;             // fragment coordinates: row group, column pair
     const int u = blockIdx.y, inst = p.inst0 + u, b = p.b, C = p.C, n1 = p.n1;
     const int rec = blockIdx.x, n_rec = gridDim.x;
@@ -206,8 +219,8 @@ decode_mq_kernel(const MqParams p) {
     // rows of this launch (rows beyond the head-instance's M are zero), natural channel order
     uint32_t qa[8][4];
     {
-        const uint32_t* q32 = reinterpret_cast<const uint32_t*>(p.q) + ((size_t)u * p.M + p.row0) * (KVR_D / 2);
-        const bool v0 = p.row0 + fg < p.M, v1 = p.row0 + fg + 8 < p.M;
+        const uint32_t* q32 = reinterpret_cast<const uint32_t*>(p.q) + ((size_t)u * p.M + rowbase) * (KVR_D / 2);
+        const bool v0 = rowbase + fg < p.M, v1 = rowbase + fg + 8 < p.M;
 #pragma unroll
         for (int s = 0; s < 8; ++s) {
             qa[s][0] = v0 ? to_h2<T>(__ldg(q32 + (size_t)fg * 64 + 8 * s + ft)) : 0u;
@@ -220,7 +233,7 @@ decode_mq_kernel(const MqParams p) {
     int vis[2];
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-        const int r = p.row0 + fg + 8 * h;
+        const int r = rowbase + fg + 8 * h;
         const int t = r % p.Qn;
         vis[h] = p.causal ? p.R - p.Qn + t + 1 : p.R;
     }
@@ -231,41 +244,46 @@ decode_mq_kernel(const MqParams p) {
 #pragma unroll
         for (int k = 0; k < 4; ++k) O[nt][k] = 0.f;
 
-    const uint32_t tile_hi = smem_s + L.tiles + (uint32_t)(warp * 2 * MQ_TILE_BYTES), tile_lo = tile_hi + MQ_TILE_BYTES;
+    const uint32_t tile_hi = smem_s + L.tiles + (uint32_t)team * 2u * TEAM_TILE_BYTES, tile_lo = tile_hi + TEAM_TILE_BYTES;
     // this lane's row address for the 8 x 8 matrix loads (matrix lane / 8, row lane % 8)
     const uint32_t ldsm_off = (uint32_t)((lane & 7) * MQ_PITCH + (lane >> 3) * 16);
 
     // S = Q K^T over the tile (hi, and lo when the tile has one), softmax step, weights as A fragments.
-    // pos[h][k]: row position in the storage of the token in column 2 ft + k (compressed tokens: -1),
-    // live: bit s set = tile slot s holds a token.
-    uint32_t pa_hi[2], pa_lo[2];
-    auto qk_softmax = [&](bool with_lo, unsigned live, int pos0, int pos1) {
-        float c[4] = {0.f, 0.f, 0.f, 0.f};
+    // live: bit s set = tile slot s holds a token; row_base >= 0: slot s is row row_base + s of the
+    // storage (a retained row: the mask among the queries' own tokens applies), else a compressed token.
+    uint32_t pa_hi[MT][2], pa_lo[MT][2];                  // per 8 tokens: rows fg | fg + 8, columns 2 ft, 2 ft + 1
+    auto qk_softmax = [&](bool with_lo, unsigned live, int row_base) {
+        float c[MT][4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            uint32_t r[4];
-            ldsm4(tile_hi + ldsm_off + j * 64, r);
-            mma_k16(c, qa[2 * j], r[0], r[1]);
-            mma_k16(c, qa[2 * j + 1], r[2], r[3]);
-        }
-        if (with_lo) {
+        for (int nt = 0; nt < MT; ++nt) {
+            c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 uint32_t r[4];
-                ldsm4(tile_lo + ldsm_off + j * 64, r);
-                mma_k16(c, qa[2 * j], r[0], r[1]);
-                mma_k16(c, qa[2 * j + 1], r[2], r[3]);
+                ldsm4(tile_hi + (uint32_t)(nt * MQ_TILE_BYTES) + ldsm_off + j * 64, r);
+                mma_k16(c[nt], qa[2 * j], r[0], r[1]);
+                mma_k16(c[nt], qa[2 * j + 1], r[2], r[3]);
+            }
+            if (with_lo) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint32_t r[4];
+                    ldsm4(tile_lo + (uint32_t)(nt * MQ_TILE_BYTES) + ldsm_off + j * 64, r);
+                    mma_k16(c[nt], qa[2 * j], r[0], r[1]);
+                    mma_k16(c[nt], qa[2 * j + 1], r[2], r[3]);
+                }
             }
         }
-        float s[4];
+        float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const int col = 2 * ft + (k & 1), h = k >> 1;
-            const int pos = (k & 1) ? pos1 : pos0;
-            const bool ok = ((live >> col) & 1u) && (pos < vis[h]);
-            s[k] = ok ? c[k] * p.scale_log2e : -INFINITY;
-        }
-        float mx[2] = {fmaxf(s[0], s[1]), fmaxf(s[2], s[3])};
+        for (int nt = 0; nt < MT; ++nt)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int col = 8 * nt + 2 * ft + (k & 1), h = k >> 1;
+                const bool ok = ((live >> col) & 1u) && (row_base < 0 || row_base + col < vis[h]);
+                c[nt][k] = ok ? c[nt][k] * p.scale_log2e : -INFINITY;
+                mx[h] = fmaxf(mx[h], c[nt][k]);
+            }
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             mx[h] = fmaxf(mx[h], __shfl_xor_sync(FULL, mx[h], 1));
@@ -282,77 +300,111 @@ decode_mq_kernel(const MqParams p) {
             m_run[0] = n0;
             m_run[1] = n1_;
         }
-        float pr[4];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) pr[k] = ex2(s[k] - m_run[k >> 1]);
-        l_run[0] += pr[0] + pr[1];
-        l_run[1] += pr[2] + pr[3];
-        split2(pr[0], pr[1], pa_hi[0], pa_lo[0]);
-        split2(pr[2], pr[3], pa_hi[1], pa_lo[1]);
-    };
-    // O += P V over the tile
-    auto pv = [&](bool with_lo) {
+        for (int nt = 0; nt < MT; ++nt) {
+            float pr[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            uint32_t r[4];
-            ldsm4_t(tile_hi + ldsm_off + j * 64, r);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                mma_k8(O[4 * j + i], pa_hi[0], pa_hi[1], r[i]);
-                mma_k8(O[4 * j + i], pa_lo[0], pa_lo[1], r[i]);
-            }
+            for (int k = 0; k < 4; ++k) pr[k] = ex2(c[nt][k] - m_run[k >> 1]);
+            l_run[0] += pr[0] + pr[1];
+            l_run[1] += pr[2] + pr[3];
+            split2(pr[0], pr[1], pa_hi[nt][0], pa_lo[nt][0]);
+            split2(pr[2], pr[3], pa_hi[nt][1], pa_lo[nt][1]);
         }
-        if (with_lo) {
+    };
+    // O += P V over the tile: 8 tokens per multiply (MT = 1) or 16 (two adjacent groups of 8 form the
+    // k dimension: their weight fragments are the four A registers as they stand)
+    auto pv = [&](bool with_lo) {
+        if constexpr (MT == 1) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 uint32_t r[4];
-                ldsm4_t(tile_lo + ldsm_off + j * 64, r);
+                ldsm4_t(tile_hi + ldsm_off + j * 64, r);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) mma_k8(O[4 * j + i], pa_hi[0], pa_hi[1], r[i]);
+                for (int i = 0; i < 4; ++i) {
+                    mma_k8(O[4 * j + i], pa_hi[0][0], pa_hi[0][1], r[i]);
+                    mma_k8(O[4 * j + i], pa_lo[0][0], pa_lo[0][1], r[i]);
+                }
+            }
+            if (with_lo) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint32_t r[4];
+                    ldsm4_t(tile_lo + ldsm_off + j * 64, r);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) mma_k8(O[4 * j + i], pa_hi[0][0], pa_hi[0][1], r[i]);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int ks = 0; ks < MT / 2; ++ks) {
+                const uint32_t ah[4] = {pa_hi[2 * ks][0], pa_hi[2 * ks][1], pa_hi[2 * ks + 1][0], pa_hi[2 * ks + 1][1]};
+                const uint32_t al[4] = {pa_lo[2 * ks][0], pa_lo[2 * ks][1], pa_lo[2 * ks + 1][0], pa_lo[2 * ks + 1][1]};
+                const uint32_t t0 = (uint32_t)(2 * ks * MQ_TILE_BYTES) + ldsm_off, t1 = t0 + MQ_TILE_BYTES;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint32_t r0[4], r1[4];
+                    ldsm4_t(tile_hi + t0 + j * 64, r0);
+                    ldsm4_t(tile_hi + t1 + j * 64, r1);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        mma_k16(O[4 * j + i], ah, r0[i], r1[i]);
+                        mma_k16(O[4 * j + i], al, r0[i], r1[i]);
+                    }
+                }
+                if (with_lo) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        uint32_t r0[4], r1[4];
+                        ldsm4_t(tile_lo + t0 + j * 64, r0);
+                        ldsm4_t(tile_lo + t1 + j * 64, r1);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) mma_k16(O[4 * j + i], ah, r0[i], r1[i]);
+                    }
+                }
             }
         }
     };
 
     // ---------------------------------------------------------------- retained rows (exact keys, values)
     {
-        const int n = r_end - r_begin, per = (n + MQ_WARPS - 1) / MQ_WARPS;
-        const int w0 = r_begin + min(warp * per, n), w1 = r_begin + min((warp + 1) * per, n);
+        const int n = r_end - r_begin, per = (n + NTEAMS - 1) / NTEAMS;
+        const int w0 = r_begin + min(team * per, n), w1 = r_begin + min((team + 1) * per, n);
         const uint2* Kr = p.Kr + (size_t)u * p.R * 32 + lg;
         const uint2* Vr = p.Vr + (size_t)u * p.R * 32 + lg;
-        for (int base = w0; base < w1; base += MQ_TILE) {
-            const int nl = min(MQ_TILE, w1 - base);
-            const unsigned live = (1u << nl) - 1u;
-            uint2 x[4][2];
+        for (int base = w0; base < w1; base += TT) {
+            const int nl = min(TT, w1 - base);
+            const unsigned live = nl >= 32 ? 0xFFFFFFFFu : (1u << nl) - 1u;
+            uint2 x[TPH][2];
 #pragma unroll
-            for (int it = 0; it < 4; ++it) {
-                const int slot = 2 * it + gw, row = base + (slot < nl ? slot : 0);
+            for (int it = 0; it < TPH; ++it) {
+                const int slot = 8 * wt + 2 * it + gw, row = base + (slot < nl ? slot : 0);
                 x[it][0] = Kr[(size_t)row * 32];
                 x[it][1] = Kr[(size_t)row * 32 + 16];
             }
 #pragma unroll
-            for (int it = 0; it < 4; ++it) {
-                const uint32_t dst = tile_hi + (uint32_t)((2 * it + gw) * MQ_PITCH + lg * 8);
+            for (int it = 0; it < TPH; ++it) {
+                const uint32_t dst = tile_hi + (uint32_t)((8 * wt + 2 * it + gw) * MQ_PITCH + lg * 8);
                 sts64(dst, to_h2<T>(x[it][0].x), to_h2<T>(x[it][0].y));
                 sts64(dst + 128, to_h2<T>(x[it][1].x), to_h2<T>(x[it][1].y));
             }
 #pragma unroll
-            for (int it = 0; it < 4; ++it) {                     // the values are on their way while the keys are used
-                const int slot = 2 * it + gw, row = base + (slot < nl ? slot : 0);
+            for (int it = 0; it < TPH; ++it) {                   // the values are on their way while the keys are used
+                const int slot = 8 * wt + 2 * it + gw, row = base + (slot < nl ? slot : 0);
                 x[it][0] = Vr[(size_t)row * 32];
                 x[it][1] = Vr[(size_t)row * 32 + 16];
             }
-            __syncwarp();
-            qk_softmax(false, live, base + 2 * ft, base + 2 * ft + 1);
-            __syncwarp();
+            team_sync();
+            qk_softmax(false, live, base);
+            team_sync();
 #pragma unroll
-            for (int it = 0; it < 4; ++it) {
-                const uint32_t dst = tile_hi + (uint32_t)((2 * it + gw) * MQ_PITCH + lg * 8);
+            for (int it = 0; it < TPH; ++it) {
+                const uint32_t dst = tile_hi + (uint32_t)((8 * wt + 2 * it + gw) * MQ_PITCH + lg * 8);
                 sts64(dst, to_h2<T>(x[it][0].x), to_h2<T>(x[it][0].y));
                 sts64(dst + 128, to_h2<T>(x[it][1].x), to_h2<T>(x[it][1].y));
             }
-            __syncwarp();
+            team_sync();
             pv(false);
-            __syncwarp();
+            team_sync();
         }
     }
 
@@ -388,11 +440,11 @@ decode_mq_kernel(const MqParams p) {
             for (int i = tid; i < len; i += MQ_THREADS) s_list[i] = clist[cb + i];
             __syncthreads();
         }
-        // the warp's tokens, in two halves: one per group of 16 lanes
-        const int per = (len + MQ_WARPS - 1) / MQ_WARPS;
-        const int w0 = min(warp * per, len), w1 = min((warp + 1) * per, len);
-        const int half = (w1 - w0 + 1) / 2;
-        const int g_begin = gw ? w0 + half : w0, g_cnt = gw ? (w1 - w0 - half) : half;
+        // the team's tokens, one contiguous part per group of 16 lanes (2 MT groups)
+        const int per = (len + NTEAMS - 1) / NTEAMS;
+        const int w0 = min(team * per, len), w1 = min((team + 1) * per, len);
+        const int half = (w1 - w0 + 2 * MT - 1) / (2 * MT);                  // tokens per group (the last groups may have fewer)
+        const int g_begin = w0 + min(hw * half, w1 - w0), g_cnt = min(half, w1 - w0 - min(hw * half, w1 - w0));
         float k0[8], v0[8];
 #pragma unroll
         for (int x = 0; x < 8; ++x) { k0[x] = 0.f; v0[x] = 0.f; }
@@ -402,21 +454,23 @@ decode_mq_kernel(const MqParams p) {
             fetch_half(ringK, g0K, c0, 0u);
             fetch_half(ringV, g0V, c0, 0u);
         }
-        for (int base = 0; base < half; base += 4) {             // 4 tokens per group and tile
+        for (int base = 0; base < half; base += TPH) {           // TPH tokens per group and tile
             unsigned live = 0u;
 #pragma unroll
-            for (int it = 0; it < 4; ++it) {
-                if (base + it < half) live |= 1u << (2 * it);
-                if (base + it < w1 - w0 - half) live |= 2u << (2 * it);
+            for (int h = 0; h < 2 * MT; ++h) {
+                const int cnt_h = min(half, w1 - w0 - min(h * half, w1 - w0));
+#pragma unroll
+                for (int it = 0; it < TPH; ++it)
+                    if (base + it < cnt_h) live |= 1u << (8 * (h >> 1) + 2 * it + (h & 1));
             }
             // ---- keys of the tile (Algorithm 2 on the key halves)
 #pragma unroll 1
-            for (int it = 0; it < 4; ++it) {
+            for (int it = 0; it < TPH; ++it) {
                 const bool lv = base + it < g_cnt;
                 const uint2 e = lds64(list_s + (uint32_t)(lv ? g_begin + base + it : 0) * 8u);
                 if (lv && ((e.y & KVR_CL_FLAG) || base + it == 0)) switch_run(k0, ringK, g0K, e.x >> KVR_CL_NEXT_SHIFT);
                 const uint32_t a1 = lane_cells + (e.x & 0xFFu) * MQ_CELLB, a2 = lane_cells + ((e.x >> 8) & 0xFFu) * MQ_CELLB;
-                const uint32_t dst = (uint32_t)((2 * it + gw) * MQ_PITCH + lg * 8);
+                const uint32_t dst = (uint32_t)((8 * wt + 2 * it + gw) * MQ_PITCH + lg * 8);
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     const float4 kb = lds128(a1 + c * 256), kc = lds128(a2 + c * 256);
@@ -429,19 +483,19 @@ decode_mq_kernel(const MqParams p) {
                     sts64(tile_lo + dst + c * 128, l0, l1);
                 }
             }
-            __syncwarp();
-            qk_softmax(true, live, -1, -1);
-            __syncwarp();
+            team_sync();
+            qk_softmax(true, live, -1);
+            team_sync();
             // ---- values of the tile; g_0 is applied to the median (med(g0 a, g1 b, g2 c) = g0 med(a, g0 g1 b, g0 g2 c))
 #pragma unroll 1
-            for (int it = 0; it < 4; ++it) {
+            for (int it = 0; it < TPH; ++it) {
                 const bool lv = base + it < g_cnt;
                 const uint2 e = lds64(list_s + (uint32_t)(lv ? g_begin + base + it : 0) * 8u);
                 if (lv && ((e.y & KVR_CL_FLAG) || base + it == 0)) switch_run(v0, ringV, g0V, e.x >> KVR_CL_NEXT_SHIFT);
                 const uint32_t a1 = lane_cells + (e.x & 0xFFu) * MQ_CELLB + MQ_HALFB, a2 = lane_cells + ((e.x >> 8) & 0xFFu) * MQ_CELLB + MQ_HALFB;
                 const float s0 = (e.y & (1u << KVR_CL_SIGN_SHIFT)) ? -1.f : 1.f;
                 const float s01 = (e.y & (2u << KVR_CL_SIGN_SHIFT)) ? -1.f : 1.f, s02 = (e.y & (4u << KVR_CL_SIGN_SHIFT)) ? -1.f : 1.f;
-                const uint32_t dst = (uint32_t)((2 * it + gw) * MQ_PITCH + lg * 8);
+                const uint32_t dst = (uint32_t)((8 * wt + 2 * it + gw) * MQ_PITCH + lg * 8);
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     const float4 vb = lds128(a1 + c * 256), vc = lds128(a2 + c * 256);
@@ -454,9 +508,9 @@ decode_mq_kernel(const MqParams p) {
                     sts64(tile_lo + dst + c * 128, l0, l1);
                 }
             }
-            __syncwarp();
+            team_sync();
             pv(true);
-            __syncwarp();
+            team_sync();
         }
     }
     asm volatile("cp.async.wait_all;\n" ::: "memory");
@@ -484,21 +538,22 @@ decode_mq_kernel(const MqParams p) {
     __syncthreads();
     {
         const float* scr = reinterpret_cast<const float*>(smem + L.cells);
-        float* part = p.part + ((size_t)u * n_rec + rec) * MQ_ROWS * PART;
-        for (int idx = tid; idx < MQ_ROWS * KVR_D; idx += MQ_THREADS) {
-            const int r = idx >> 7, d = idx & (KVR_D - 1);
+        float* part = p.part + ((size_t)u * n_rec + rec) * ROWS_L * PART;
+        for (int idx = tid; idx < ROWS_L * KVR_D; idx += MQ_THREADS) {
+            const int rl = idx >> 7, d = idx & (KVR_D - 1);
+            const int mt = rl / MQ_ROWS, r = rl % MQ_ROWS;              // the teams' warps that hold these 16 rows: t * MT + mt
             float M = M_EMPTY;
 #pragma unroll
-            for (int w = 0; w < MQ_WARPS; ++w) M = fmaxf(M, scr[(w * MQ_ROWS + r) * PART + KVR_D]);
+            for (int t = 0; t < NTEAMS; ++t) M = fmaxf(M, scr[((t * MT + mt) * MQ_ROWS + r) * PART + KVR_D]);
             float Ls = 0.f, Os = 0.f;
 #pragma unroll
-            for (int w = 0; w < MQ_WARPS; ++w) {
-                const float f = ex2(scr[(w * MQ_ROWS + r) * PART + KVR_D] - M);
-                Ls += scr[(w * MQ_ROWS + r) * PART + KVR_D + 1] * f;
-                Os += scr[(w * MQ_ROWS + r) * PART + d] * f;
+            for (int t = 0; t < NTEAMS; ++t) {
+                const float f = ex2(scr[((t * MT + mt) * MQ_ROWS + r) * PART + KVR_D] - M);
+                Ls += scr[((t * MT + mt) * MQ_ROWS + r) * PART + KVR_D + 1] * f;
+                Os += scr[((t * MT + mt) * MQ_ROWS + r) * PART + d] * f;
             }
-            part[r * PART + d] = Os;
-            if (d == 0) { part[r * PART + KVR_D] = M; part[r * PART + KVR_D + 1] = Ls; }
+            part[rl * PART + d] = Os;
+            if (d == 0) { part[rl * PART + KVR_D] = M; part[rl * PART + KVR_D + 1] = Ls; }
         }
     }
     // ---------------------------------------------------------------- last CTA of the head-instance merges
@@ -512,15 +567,15 @@ decode_mq_kernel(const MqParams p) {
     __syncthreads();
     if (!*s_flag) return;
     __threadfence();
-    const float* recs = p.part + (size_t)u * n_rec * MQ_ROWS * PART;
-    for (int idx = tid; idx < MQ_ROWS * KVR_D; idx += MQ_THREADS) {
+    const float* recs = p.part + (size_t)u * n_rec * ROWS_L * PART;
+    for (int idx = tid; idx < ROWS_L * KVR_D; idx += MQ_THREADS) {
         const int r = idx >> 7, d = idx & (KVR_D - 1);
         if (p.row0 + r >= p.M) continue;
         float M = M_EMPTY;
-        for (int c = 0; c < n_rec; ++c) M = fmaxf(M, __ldcg(recs + ((size_t)c * MQ_ROWS + r) * PART + KVR_D));
+        for (int c = 0; c < n_rec; ++c) M = fmaxf(M, __ldcg(recs + ((size_t)c * ROWS_L + r) * PART + KVR_D));
         float Ls = 0.f, Os = 0.f;
         for (int c = 0; c < n_rec; ++c) {                  // fixed order: the result does not depend on timing
-            const float* pr = recs + ((size_t)c * MQ_ROWS + r) * PART;
+            const float* pr = recs + ((size_t)c * ROWS_L + r) * PART;
             const float f = ex2(__ldcg(pr + KVR_D) - M);
             Ls += __ldcg(pr + KVR_D + 1) * f;
             Os += __ldcg(pr + d) * f;
@@ -555,7 +610,7 @@ bool kvr_decode_mq_plan(const kvr_sketch* sk, int n_inst, int N, int R, int* S_o
     return *smem_out <= MQ_SMEM_LIMIT;
 }
 
-size_t kvr_decode_mq_ws_bytes(int n_inst, int records) { return sizeof(float) * (size_t)n_inst * records * MQ_ROWS * kvr_dec::PART; }
+size_t kvr_decode_mq_ws_bytes(int n_inst, int records) { return sizeof(float) * (size_t)n_inst * records * 4 * MQ_ROWS * kvr_dec::PART; }
 
 cudaError_t kvr_launch_decode_mq(kvr_sketch* sk, int inst0, int n_inst, int rows, const void* q, const void* Kr, const void* Vr,
                                  int n_queries, int causal, float scale, float* out, int S, int lcap, size_t smem, float* part,
@@ -586,16 +641,22 @@ cudaError_t kvr_launch_decode_mq(kvr_sketch* sk, int inst0, int n_inst, int rows
     p.zero = 0u;
     p.scale_log2e = scale * 1.4426950408889634f;
     const bool f16 = sk->d.kv_dtype == KVR_F16;
-    auto kern = f16 ? decode_mq_kernel<__half> : decode_mq_kernel<__nv_bfloat16>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
     const dim3 grid(sk->C * sk->C * S, n_inst);
-    for (int row0 = 0; row0 < p.M; row0 += MQ_ROWS) {       // 16 query rows per launch
+    // 64, 32 or 16 query rows per launch: as many as are left
+    for (int row0 = 0; row0 < p.M;) {
+        const int left = p.M - row0, mt = left > 32 ? 4 : left > 16 ? 2 : 1;
+        void (*kern)(const MqParams) =
+            mt == 4 ? (f16 ? decode_mq_kernel<__half, 4> : decode_mq_kernel<__nv_bfloat16, 4>)
+          : mt == 2 ? (f16 ? decode_mq_kernel<__half, 2> : decode_mq_kernel<__nv_bfloat16, 2>)
+                    : (f16 ? decode_mq_kernel<__half, 1> : decode_mq_kernel<__nv_bfloat16, 1>);
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
         p.row0 = row0;
         kern<<<grid, MQ_THREADS, smem, st>>>(p);
         sk->launches += 1;
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
+        row0 += MQ_ROWS * mt;
     }
     return cudaSuccess;
 }

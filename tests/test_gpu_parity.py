@@ -465,9 +465,11 @@ def test_append_runs_algorithm_3_over_several_slack_periods(which, dtype, one_ca
 
 @pytest.mark.parametrize("Qn,dtype,causal,b,N0,R", [
     (1, F16, True, 20, 1200, 150),          # one query: the single-query result
-    (4, F16, True, 20, 1200, 150),          # 16 query rows = one launch
+    (4, F16, True, 20, 1200, 150),          # 16 query rows: every warp on its own
     (4, BF16, False, 20, 1200, 150),
-    (16, F16, True, 200, 5000, 900),        # 64 query rows = four launches; 4 x 4 classes
+    (16, F16, True, 200, 5000, 900),        # 64 query rows: teams of four warps share a tile; 4 x 4 classes
+    (8, BF16, True, 64, 3000, 400),         # 32 query rows: teams of two
+    (17, F16, False, 33, 2000, 300),        # 68 query rows: a launch of 64 and one of 16 (4 rows used)
     (16, BF16, True, 20, 700, 100),
     (3, F16, True, 37, 900, 0),             # nothing retained but the queries' own tokens; 12 rows (padded to 16)
 ])
