@@ -60,7 +60,7 @@ __host__ __device__ inline MqLayout mq_layout(int n1, int lcap) {
     int o = 0;
     L.ctrl = o;  o += 32;                                  // last-arriver flag; staging mbarriers at +16, +24
     L.ring = o;  o += MQ_GROUPS * 2 * MQ_HALFB;            // per group: key half and value half of a row-0 cell in flight
-    L.tiles = o; o += MQ_WARPS * 2 * MQ_TILE_BYTES;        // per warp: hi tile, lo tile
+    L.tiles = o; o += MQ_WARPS * 2 * MQ_TILE_BYTES;        // per team of MT warps: hi tile, lo tile of 8 MT tokens
     L.list = o;  o += ((lcap + 2) * 8 + 15) & ~15;
     L.cells = o; o += 2 * n1 * MQ_CELLB;                   // row-1 slice, row-2 slice (later: the warps' records)
     L.total = o;
