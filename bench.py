@@ -271,7 +271,7 @@ def run_gpu(args, w, rank, world, local):
                  "smem": smem_bytes / lds_peak * 1e6}
     binding = {"nearest_ceiling": max(floors_us, key=floors_us.get),
                "floor_us": {k: round(v, 2) for k, v in floors_us.items()},
-               "note": "the launch also spends instruction issue slots around these; see DESIGN.md section 8"}
+               "note": "the launch also spends instruction issue slots around these: at its instruction count the issue floor alone is about 22 us"}
     # ---- same decode work as ONE launch over all layers per decode step (upper bound on launch shape) ----
     batched = None
     if L > 1:
