@@ -473,6 +473,40 @@ def test_swap_with_rate_one_leaves_the_top_scores_in_the_candidate_part():
     np.testing.assert_array_equal(ts[vague], tok[vague])
 
 
+@pytest.mark.parametrize("seed,rate,limit", [(210, 1.0, 10 ** 6), (211, 1.1, 10 ** 6), (212, 1.5, 7), (213, 1.0, 5),
+                                             (214, 1.1, 10 ** 6), (215, 2.0, 10 ** 6)])
+def test_swap_loop_pairs_sorted_candidates_with_sorted_vague_tokens(seed, rate, limit):
+    """With ReplaceRate >= 1 and scores >= 0 the loop never touches a token twice, so its k-th exchange is
+    the k-th worst candidate (score, then token index) against the k-th best vague token (score
+    descending, then token index) of the lists as they stand at entry, until the first pair that fails
+    C.Min * ReplaceRate < V.Max.  Written out here with two sorts, scores with many ties included, and
+    compared with the loop taken one exchange at a time: which rows hold which tokens and scores."""
+    K, V, seeds, b, c, tok, rows = _swap_case(seed)
+    R, n_recent, N = 12, 3, 48
+    rng = np.random.default_rng(seed)
+    tok = (rng.integers(0, 6, size=N) / 4.0).astype(np.float32)                # few distinct values: ties everywhere
+    rows = (rng.integers(0, 6, size=R) / 4.0).astype(np.float32)
+    ret0 = c["ret_idx"][0]
+    Kr, Vr, ret, rs, ts, cells, n = orc.swap(c["Kr"][0], c["Vr"][0], ret0, rows, tok, c["cells"][0], n_recent, rate, limit, seeds)
+    n_cand = R - n_recent
+    cand = sorted(range(n_cand), key=lambda r: (rows[r], ret0[r]))              # rows, worst first
+    vague = sorted(np.setdiff1d(np.arange(N), ret0), key=lambda J: (-float(tok[J]), J))     # tokens, best first
+    want_ret, want_rs, want_ts = ret0.copy(), rows.copy(), tok.copy()
+    k = 0
+    while k < min(limit, n_cand, len(vague)):
+        r, J = cand[k], vague[k]
+        if not (np.float32(rows[r] * np.float32(rate)) < tok[J]):
+            break
+        want_ts[ret0[r]] = rows[r]
+        want_ret[r], want_rs[r] = J, tok[J]
+        k += 1
+    assert n == k
+    np.testing.assert_array_equal(ret, want_ret)
+    np.testing.assert_array_equal(rs, want_rs)
+    left = np.setdiff1d(np.arange(N), want_ret)
+    np.testing.assert_array_equal(ts[left], want_ts[left])
+
+
 def test_swap_under_injective_hashing_revives_exactly_and_keeps_the_sketch_consistent():
     """One cell per token (no collisions): V.Query returns the original vectors, so a revived row is
     the token's own K, V, and after Delete + Insert the cells equal a sketch built directly from the
