@@ -223,9 +223,9 @@ __device__ int swap_loop_in_order(const SwapArgs& A, T* Kr, T* Vr, int done, int
 // The K smallest of n distinct 64-bit keys (hi(i) << 32 | lo(i)), ascending: their positions go to
 // out_pos[0..K).  All 1024 threads call it.  hi(i) is cheap (the caller keeps the score images in
 // shared memory where they fit); lo(i) reads global memory.
-//   1. Every thread takes the smallest high word of its own keys (i = tid, tid + 1024, ...); the
-//      K-th smallest of these 1024 minima, U, bounds the K-th key from above, because K different
-//      keys lie at or below it.
+//   1. Every thread takes the smallest high word of its own keys (i = tid, tid + 1024, ...); a value U
+//      with at least K of these 1024 minima at or below it bounds the K-th key from above, because K
+//      different keys lie at or below it.
 //   2. The keys with high word <= U are collected (normally a small multiple of K) and sorted.
 //   3. Should they not fit (more than SW_M: many equal scores), the K-th key is found bit by bit
 //      instead: T grows from the top bit down while fewer than K keys lie below it, one count over
@@ -247,18 +247,31 @@ template <class HiFn, class LoFn>
 __device__ void swap_select(int n, int K, HiFn hi, LoFn lo, unsigned long long* s_lk, int* s_lp, int* s_cnt, int* s_misc,
                             int* out_pos) {
     const int tid = threadIdx.x, lane = tid & 31;
-    // ---- 1. the K-th smallest of the threads' minima
+    // ---- 1. a bound from the threads' minima: every warp sorts its 32 minima (shuffles only) and names its
+    // t-th smallest, t = ceil(K / 32); the largest of the 32 warps' answers has at least 32 t >= K keys at or
+    // below it.  (One barrier instead of a bit-by-bit search for the exact K-th minimum; a little looser.)
     uint32_t U;
     {
         uint32_t mn = 0xFFFFFFFFu;
         for (int i = tid; i < n; i += 1024) mn = min(mn, hi(i));
         if (tid == 0) s_misc[2] = 0;
-        // U = the largest value with fewer than K minima below it, bit by bit (one barrier per bit)
-        U = 0u;
-        for (int bit = 31; bit >= 0; --bit) {
-            const uint32_t trial = U | (1u << bit);
-            if (__syncthreads_count(mn < trial) < K) U = trial;
-        }
+#pragma unroll
+        for (int k = 2; k <= 32; k <<= 1)
+#pragma unroll
+            for (int j = k >> 1; j > 0; j >>= 1) {
+                const uint32_t o = __shfl_xor_sync(0xFFFFFFFFu, mn, j);
+                const bool up = ((lane & k) == 0) == ((lane & j) == 0);      // this lane keeps the smaller of the two
+                mn = up ? min(mn, o) : max(mn, o);
+            }
+        const int t = (K + 31) >> 5;                              // 1 .. SW_K / 32
+        const uint32_t mine = __shfl_sync(0xFFFFFFFFu, mn, t - 1);
+        if (lane == 0) s_cnt[tid >> 5] = (int)mine;
+        __syncthreads();
+        uint32_t v = (uint32_t)s_cnt[lane];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+        U = v;
+        __syncthreads();
     }
     // ---- 2. the keys at or below U (a warp reserves its places with one addition)
     for (int base = 0; base < n; base += 1024) {
@@ -323,24 +336,51 @@ __device__ void swap_select(int n, int K, HiFn hi, LoFn lo, unsigned long long* 
         M = min(s_misc[2], SW_M);
         __syncthreads();
     }
-    int P = 2;
+    int P = 32;
     while (P < M) P <<= 1;
     for (int i = M + tid; i < P; i += 1024) { s_lk[i] = ~0ull; s_lp[i] = 0; }
     __syncthreads();
-    for (int k = 2; k <= P; k <<= 1)
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int i = tid; i < P; i += 1024) {
-                const int x = i ^ j;
-                if (x > i) {
-                    const unsigned long long ka = s_lk[i], kb = s_lk[x];
-                    if ((ka > kb) == ((i & k) == 0)) {
-                        s_lk[i] = kb; s_lk[x] = ka;
-                        const int pa = s_lp[i]; s_lp[i] = s_lp[x]; s_lp[x] = pa;
+    if (P <= 1024) {
+        // one key per thread: exchanges between lanes of a warp go through shuffles, the others through
+        // shared memory with a barrier (10 of the 45 steps of a sort of 512)
+        unsigned long long key = tid < P ? s_lk[tid] : ~0ull;
+        int pos = tid < P ? s_lp[tid] : 0;
+        for (int k = 2; k <= P; k <<= 1)
+            for (int j = k >> 1; j > 0; j >>= 1) {
+                unsigned long long ok;
+                int op;
+                if (j >= 32) {
+                    __syncthreads();                              // (everybody has read the previous exchange)
+                    if (tid < P) { s_lk[tid] = key; s_lp[tid] = pos; }
+                    __syncthreads();
+                    ok = tid < P ? s_lk[tid ^ j] : ~0ull;
+                    op = tid < P ? s_lp[tid ^ j] : 0;
+                } else {
+                    ok = __shfl_xor_sync(0xFFFFFFFFu, key, j);
+                    op = __shfl_xor_sync(0xFFFFFFFFu, pos, j);
+                }
+                const bool keep_small = ((tid & k) == 0) == ((tid & j) == 0);
+                if (keep_small ? ok < key : ok > key) { key = ok; pos = op; }
+            }
+        __syncthreads();
+        if (tid < P) { s_lk[tid] = key; s_lp[tid] = pos; }
+        __syncthreads();
+    } else {
+        for (int k = 2; k <= P; k <<= 1)
+            for (int j = k >> 1; j > 0; j >>= 1) {
+                for (int i = tid; i < P; i += 1024) {
+                    const int x = i ^ j;
+                    if (x > i) {
+                        const unsigned long long ka = s_lk[i], kb = s_lk[x];
+                        if ((ka > kb) == ((i & k) == 0)) {
+                            s_lk[i] = kb; s_lk[x] = ka;
+                            const int pa = s_lp[i]; s_lp[i] = s_lp[x]; s_lp[x] = pa;
+                        }
                     }
                 }
+                __syncthreads();
             }
-            __syncthreads();
-        }
+    }
     if (tid < K) out_pos[tid] = s_lp[tid];
     __syncthreads();
 }
